@@ -1,0 +1,348 @@
+#!/usr/bin/env python
+"""Benchmark of the token-routing step (one step = one tlr_route call over one batch).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl reference]
+
+Prints ONE JSON line.  The default workload is the batched-decode configuration
+(256 sessions x 1 token, d=896, V=151936, tau=0.5) on synthetic seeded inputs.
+With --gpus N > 1 (launched under torch.distributed.run) every rank routes its own
+batch of the same size with its own copy of W (rows are independent units, so the
+path shards with no data-path collective): weak scaling, time = max over ranks.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import sys
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import tlr_synth as S  # noqa: E402
+
+METRIC = "routed-path tokens/s (rows through tlr_route per second, all six outputs)"
+UNIT = "tokens/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reported against the HBM roofline
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return json.load(f), "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def algorithmic_bytes(n, d, V):
+    """W once + h once + the six outputs (17 bytes per row + the count)."""
+    return 2 * V * d + 2 * n * d + 17 * n + 4
+
+
+def algorithmic_flops(n, d, V):
+    return 2 * n * d * V
+
+
+class ClockSampler:
+    """Polls NVML (SM clock, power, throttle reasons) from the host while the GPU works."""
+
+    def __init__(self, index):
+        self.samples = []
+        self.reasons = set()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.max_mhz = None
+
+    def sample(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        try:
+            self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+            r = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+            names = {"hw_slowdown": nv.nvmlClocksEventReasonHwSlowdown,
+                     "hw_thermal_slowdown": nv.nvmlClocksEventReasonHwThermalSlowdown,
+                     "sw_thermal_slowdown": nv.nvmlClocksEventReasonSwThermalSlowdown,
+                     "sw_power_cap": nv.nvmlClocksEventReasonSwPowerCap}
+            for k, bit in names.items():
+                if r & bit:
+                    self.reasons.add(k)
+        except Exception:
+            pass
+
+    def summary(self):
+        return {"sm_mhz": float(np.median(self.samples)) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def physical_gpu_index(local_rank):
+    vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+    if vis:
+        try:
+            return int(vis.split(",")[local_rank])
+        except Exception:
+            return local_rank
+    return local_rank
+
+
+def run_ours(args):
+    import paper_2504_07878_b200 as P
+    from paper_2504_07878_b200 import build
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        if world == 1 and args.gpus > 1:
+            raise SystemExit("--gpus %d needs `python -m torch.distributed.run --nproc-per-node %d`"
+                             % (args.gpus, args.gpus))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the routing path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if rank == 0:
+        build.build()
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    P.load_library()
+
+    wl = S.WORKLOADS[args.workload]
+    n, d, V = wl.n, wl.d, wl.V
+    tau = 0.5 if wl.tau is None else wl.tau
+    W_host = S.make_W(d, V, seed=0)
+    hid = S.make_h(n, d, seed=rank, W=W_host, planted_fraction=wl.planted_fraction)
+    # two device copies of W, alternated step by step: together with W > L2 this makes every
+    # step stream W from HBM rather than from whatever the previous step left in L2
+    copies = 2
+    Ws = [W_host.cuda() for _ in range(copies)]
+    routers = [P.Router(w, max_n=n) for w in Ws]
+    h_dev = hid.h.cuda()
+    plan = P.tlr_plan_query(routers[0].ctx, n)
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        routers[i % copies].route(h_dev, tau, stream)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        step(i)
+    barrier()
+
+    # ---- timed region: exactly K steps, device time between two events, clocks sampled meanwhile
+    sampler = ClockSampler(physical_gpu_index(local_rank))
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(args.steps):
+        step(i)
+    e1.record(stream)
+    while not e1.query():
+        sampler.sample()
+        time.sleep(0.002)
+    sampler.sample()
+    barrier()
+    ms_total = e0.elapsed_time(e1)
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([ms_total], device="cuda")
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_total = float(t.item())
+    status = max(P.tlr_last_device_status(r.ctx) for r in routers)
+    if status & P.TLR_DEV_WAIT_TIMEOUT:
+        raise SystemExit("device status flags raised during the timed region: %d" % status)
+    routed = int(routers[0].routed_count.item())
+
+    # ---- dominant kernel alone: the projection kernel bracketed by events inside tlr_route
+    for r in routers:
+        P.tlr_set_kernel_timing(r.ctx, True)
+    ksteps = min(args.steps, 2000)
+    for i in range(ksteps):
+        step(i)
+    torch.cuda.synchronize()
+    launches, kms = 0, 0.0
+    for r in routers:
+        ln, ms = P.tlr_read_kernel_timing(r.ctx)
+        launches += ln
+        kms += ms
+        P.tlr_set_kernel_timing(r.ctx, False)
+    kernel_ms = kms / max(launches, 1)
+
+    # ---- end to end through the host-buffer entry point (pinned host memory)
+    h_pin = hid.h.pin_memory()
+    o_tok = torch.empty(n, dtype=torch.int32).pin_memory()
+    o_conf = torch.empty(n, dtype=torch.float32).pin_memory()
+    o_ent = torch.empty(n, dtype=torch.float32).pin_memory()
+    o_mask = torch.empty(n, dtype=torch.uint8).pin_memory()
+    o_idx = torch.empty(n, dtype=torch.int32).pin_memory()
+    o_cnt = torch.zeros(1, dtype=torch.int32).pin_memory()
+    esteps = min(args.steps, 2000)
+
+    def host_step(i):
+        P.tlr_route_host(routers[i % copies].ctx, h_pin, n, tau, o_tok, o_conf, o_ent, o_mask, o_idx, o_cnt, stream)
+
+    for i in range(max(3, min(args.warmup, 20))):
+        host_step(i)
+    barrier()
+    t0 = time.perf_counter()
+    for i in range(esteps):
+        host_step(i)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    if world > 1:
+        import torch.distributed as dist
+        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        e2e_s = float(t.item())
+    e2e_routed = int(o_cnt.item())
+    h2d = n * d * 2
+    d2h = n * (4 + 4 + 4 + 1) + 4 + 4 + 4 * e2e_routed      # + status word + routed_idx[:count]
+
+    if rank != 0:
+        return
+    peaks, peak_kind = measured_peaks()
+    ms_per_step = ms_total / args.steps
+    value = world * n / (ms_per_step * 1e-3)
+    hbm_bound = n <= RIDGE_ROWS_HBM
+    if hbm_bound:
+        achieved = algorithmic_bytes(n, d, V) / (kernel_ms * 1e-3) / 1e9
+        peak = float(peaks["hbm_gbs"])
+        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s"}
+    else:
+        achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
+        peak = float(peaks.get("bf16_tflops_sustained" if ms_total > 1000 else "bf16_tflops", peaks["bf16_tflops"]))
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s"}
+    roof.update({"frac": achieved / peak, "traffic": None, "peak_source": "of " + peak_kind,
+                 "kernel": "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel",
+                 "kernel_ms": kernel_ms, "kernel_launches_timed": launches,
+                 "tensor_frac_same_launch": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
+                 float(peaks["bf16_tflops"]),
+                 "hbm_frac_same_launch": algorithmic_bytes(n, d, V) / (kernel_ms * 1e-3) / 1e9 /
+                 float(peaks["hbm_gbs"])})
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "bf16 in, fp32 accumulate and softmax statistics", "data": "synthetic",
+        "config": {"workload": "%s: n=%d rows, d=%d, V=%d, tau=%g%s" % (wl.name, n, d, V, tau,
+                                                                       ", %.0f%% planted rows" % (100 * wl.planted_fraction)
+                                                                       if wl.planted_fraction else ""),
+                   "l2": "inputs larger than L2: W is %.0f MB and two device copies of it alternate between steps"
+                         % (2 * V * d / 1e6),
+                   "path": int(plan.path), "grid": int(plan.grid), "block": int(plan.block),
+                   "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed},
+        "e2e": {"value": world * n * esteps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+                "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)"},
+        "gpu_launches": int(plan.launches) * args.steps,
+        "clocks": sampler.summary(),
+        "roofline": roof,
+    }
+    if world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, W_host, hid, tau, budget_s=15.0)
+    print(json.dumps(out))
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        ts = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        if ts:
+            return int(max(ts))
+    except Exception:
+        pass
+    return os.cpu_count() or 1
+
+
+def cpu_baseline(wl, W_host, hid, tau, budget_s):
+    """The fp64 oracle, as it stands, on a bounded sample of the workload's rows."""
+    from oracle import route_oracle as O
+    Wb = S.bf16_bits(W_host)
+    W64 = O.bf16_bits_to_f64(Wb)
+    hb = S.bf16_bits(hid.h)
+    probe = min(8, wl.n)
+    t0 = time.perf_counter()
+    O.route_oracle(hb[:probe], Wb, tau, W64=W64)
+    per_row = (time.perf_counter() - t0) / probe
+    rows = int(max(1, min(wl.n, budget_s / max(per_row, 1e-9))))
+    t0 = time.perf_counter()
+    O.route_oracle(hb[:rows], Wb, tau, W64=W64)
+    dt = time.perf_counter() - t0
+    return {"value": rows / dt, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": "first %d of %d rows of the same workload, W already widened to fp64, %.1f s"
+                      % (rows, wl.n, dt)}
+
+
+def run_reference(args):
+    """The reference arm: the CPU fp64 oracle on the same workload, a bounded sample of rows per step."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import route_oracle as O
+    wl = S.WORKLOADS[args.workload]
+    tau = 0.5 if wl.tau is None else wl.tau
+    W_host = S.make_W(wl.d, wl.V, seed=0)
+    hid = S.make_h(wl.n, wl.d, seed=0, W=W_host, planted_fraction=wl.planted_fraction)
+    Wb = S.bf16_bits(W_host)
+    W64 = O.bf16_bits_to_f64(Wb)
+    hb = S.bf16_bits(hid.h)
+    probe = min(4, wl.n)
+    t0 = time.perf_counter()
+    O.route_oracle(hb[:probe], Wb, tau, W64=W64)
+    per_row = (time.perf_counter() - t0) / probe
+    budget = 90.0 / max(1, args.steps + args.warmup)
+    rows = int(max(1, min(wl.n, budget / max(per_row, 1e-9))))
+    for i in range(args.warmup):
+        O.route_oracle(hb[:rows], Wb, tau, W64=W64)
+    t0 = time.perf_counter()
+    for i in range(args.steps):
+        O.route_oracle(hb[:rows], Wb, tau, W64=W64)
+    dt = time.perf_counter() - t0
+    value = rows * args.steps / dt
+    sample = "each step = the first %d of %d rows, W already widened to fp64" % (rows, wl.n)
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt / args.steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": "%s: n=%d rows, d=%d, V=%d, tau=%g" % (wl.name, wl.n, wl.d, wl.V, tau),
+                      "sample": sample},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=4000)
+    ap.add_argument("--warmup", type=int, default=50)
+    ap.add_argument("--workload", default="decode256", choices=sorted(S.WORKLOADS))
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

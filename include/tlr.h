@@ -1,0 +1,164 @@
+/*
+ * tlr -- token-level routing step on one NVIDIA B200 (sm_100a).
+ *
+ * For n decoding positions the library takes the small model's last-layer hidden
+ * states h[n,d] and its LM-head matrix W[V,d] and produces, without ever writing the
+ * n x V logits to memory,
+ *
+ *     token[i]      = argmax_v  z[i,v],   z[i,v] = sum_k h[i,k] W[v,k]   (lowest v on ties)
+ *     conf[i]       = max_v softmax(z[i,:])_v          (the "confidence score")
+ *     entropy[i]    = -sum_v p_v ln p_v                (nats)
+ *     route_mask[i] = conf[i] < tau ? 1 : 0            (1 = send this token to the large model)
+ *     routed_idx    = ascending list of the i with route_mask[i] = 1
+ *     routed_count  = length of that list
+ *
+ * Where this comes from in the paper ("Token Level Routing Inference System for Edge
+ * Devices", arXiv 2504.07878): Sec. 3.1 "Front End" defines the decision -- a score is
+ * computed from the small model's last-layer hidden state and the token is routed to
+ * the large model when the score falls below the threshold; Sec. 2.1 names the
+ * threshold tau; Sec. 3.3 "Backend" exposes the last-layer hidden state, which is the
+ * LM head's input; the record of Fig. 5 carries the same quantities (hidden_states,
+ * routing_threshold, current_token, per-token route flag, token_index).  The paper
+ * gives no dimensions or weights for its learned score, so the score here is the small
+ * model's own max softmax probability; entropy is reported beside it.  Batching over n
+ * positions and the index list are this library's data-parallel restatement of the
+ * paper's one-token-at-a-time loop.
+ *
+ * All pointers named *_dev are device pointers on the context's GPU; *_host are host
+ * pointers.  The library never takes ownership of a caller's buffer.  Every function
+ * returns a status code; none throws, aborts or prints.
+ */
+#ifndef TLR_H_
+#define TLR_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tlr_ctx tlr_ctx; /* opaque */
+
+typedef enum {
+  TLR_OK = 0,
+  TLR_ERR_ARG = 1,           /* null pointer, negative size, n > max_n, ... */
+  TLR_ERR_ALIGN = 2,         /* W or h not 16-byte aligned */
+  TLR_ERR_UNSUPPORTED = 3,   /* device is not sm_100, or a shape the kernels cannot address */
+  TLR_ERR_CUDA = 4,          /* a CUDA runtime/driver call failed */
+  TLR_ERR_NOMEM = 5,         /* workspace allocation failed */
+  TLR_ERR_TOO_MANY_ROWS = 6, /* n > max_n given at creation */
+  TLR_ERR_DEVICE_STATUS = 7  /* a kernel reported a fault flag (see tlr_last_device_status) */
+} tlr_status;
+
+/* Which projection kernel a call of n rows uses. */
+typedef enum {
+  TLR_PATH_AUTO = 0,   /* choose by shape (default) */
+  TLR_PATH_SIMT = 1,   /* CUDA-core kernel: any d, any V; the only path when d % 8 != 0 */
+  TLR_PATH_TC = 2      /* tcgen05 tensor-core kernel fed by TMA; needs d % 8 == 0 */
+} tlr_path;
+
+/* Launch plan of the projection kernel for a given n (for reports and tests). */
+typedef struct {
+  int32_t path;          /* tlr_path actually used */
+  int32_t grid;          /* CTAs launched */
+  int32_t block;         /* threads per CTA */
+  int32_t row_units;     /* ceil(n / rows per CTA tile) */
+  int32_t vocab_chunks;  /* partial results per row that the merge step folds */
+  int32_t smem_bytes;    /* dynamic shared memory per CTA */
+  int32_t launches;      /* kernels launched per tlr_route call */
+  int32_t reserved;
+} tlr_plan;
+
+/* Bits of the device status word (tlr_last_device_status). */
+#define TLR_DEV_WAIT_TIMEOUT 1u   /* a bounded barrier wait inside a kernel gave up */
+#define TLR_DEV_NONFINITE 2u      /* a row produced a confidence that is not a number */
+
+/*
+ * tlr_create -- bind an LM head to a context (Sec. 3.3: the head whose input is the
+ * exposed last-layer hidden state).
+ *   d, V        hidden size and vocabulary size, both > 0.
+ *   W_bf16_dev  device pointer to W, bf16, row-major [V, d] (row v = output embedding of
+ *               token v), 16-byte aligned.  BORROWED for the life of the context: the
+ *               caller keeps it allocated and unchanged; it is not copied.
+ *   max_n       largest n any later call will pass (>= 1).  Sizes the workspace.
+ *   out         receives the context.
+ * The only call that allocates device memory: the per-row partial-result workspace,
+ * a status word, and staging buffers for tlr_route_host.  Uses the current CUDA device.
+ * Errors: TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED (not an sm_100 device),
+ * TLR_ERR_NOMEM, TLR_ERR_CUDA.  On error *out is NULL and nothing is leaked.
+ */
+tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_n, tlr_ctx** out);
+
+/*
+ * tlr_route -- the routing step for n positions (Sec. 3.1 decision rule; Sec. 2.1 tau).
+ *   h_bf16_dev        bf16 row-major [n, d], 16-byte aligned, caller-owned.
+ *   n                 0 <= n <= max_n.  n == 0 writes routed_count = 0 and nothing else.
+ *   tau               threshold; not range-checked (tau <= 0 routes nothing, tau > 1 routes all).
+ *                     A row whose confidence is not a number is routed and raises
+ *                     TLR_DEV_NONFINITE.
+ *   token_dev         int32 [n]   out
+ *   conf_dev          float [n]   out
+ *   entropy_dev       float [n]   out
+ *   route_mask_dev    uint8 [n]   out, 0 or 1
+ *   routed_idx_dev    int32 [n]   out, capacity n; entries [0, routed_count) are valid and
+ *                                 ascending, the rest are left untouched
+ *   routed_count_dev  int32 [1]   out, stays on the device
+ *   cuda_stream       a cudaStream_t (NULL = legacy default stream)
+ * Enqueues its kernels on cuda_stream and returns without synchronising; outputs are
+ * valid once the stream reaches that point.  Allocates nothing.  Calls on one context
+ * share its workspace, so they must be ordered (same stream, or externally serialised).
+ * Errors (all detected on the host before any launch): TLR_ERR_ARG, TLR_ERR_ALIGN,
+ * TLR_ERR_TOO_MANY_ROWS, TLR_ERR_CUDA.
+ */
+tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
+                     int32_t* token_dev, float* conf_dev, float* entropy_dev,
+                     uint8_t* route_mask_dev, int32_t* routed_idx_dev,
+                     int32_t* routed_count_dev, void* cuda_stream);
+
+/*
+ * tlr_route_host -- the same step with HOST buffers: copies h to the device, runs
+ * tlr_route, copies the six results back, and synchronises the stream before
+ * returning.  Host buffers may be pageable or pinned (pinned is faster).  Output
+ * pointers may be NULL to skip that copy, except routed_count_host.  routed_idx_host
+ * needs capacity n; only the first *routed_count_host entries are written.
+ * Same errors as tlr_route, plus TLR_ERR_DEVICE_STATUS when a kernel raised
+ * TLR_DEV_WAIT_TIMEOUT (outputs are then not to be trusted).
+ */
+tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau,
+                          int32_t* token_host, float* conf_host, float* entropy_host,
+                          uint8_t* route_mask_host, int32_t* routed_idx_host,
+                          int32_t* routed_count_host, void* cuda_stream);
+
+/* tlr_destroy -- free the context's workspace.  W is left alone.  NULL is TLR_OK. */
+tlr_status tlr_destroy(tlr_ctx* ctx);
+
+/* Static, never-NULL description of a status code. */
+const char* tlr_status_string(tlr_status s);
+
+/*
+ * tlr_last_device_status -- read and clear the device status word (an OR of TLR_DEV_*
+ * bits raised by kernels since the last read).  Synchronises the device.
+ */
+tlr_status tlr_last_device_status(tlr_ctx* ctx, uint32_t* out_host);
+
+/* tlr_set_path -- force the projection kernel (tests, diagnostics).  TLR_ERR_UNSUPPORTED
+ * if the shape cannot run on the requested path. */
+tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path);
+
+/* tlr_plan_query -- the launch plan a call with n rows would use.  No device work. */
+tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out);
+
+/*
+ * tlr_set_kernel_timing -- when enabled, every tlr_route call brackets its projection
+ * kernel (the dominant one) with CUDA events on the call's stream.
+ * tlr_read_kernel_timing synchronises those events and returns the number of bracketed
+ * launches since the last read and their summed device time in milliseconds, then
+ * resets the tally.  At most 4096 launches are kept between reads.
+ */
+tlr_status tlr_set_kernel_timing(tlr_ctx* ctx, int32_t enabled);
+tlr_status tlr_read_kernel_timing(tlr_ctx* ctx, int32_t* launches_out, float* total_ms_out);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TLR_H_ */

@@ -128,6 +128,12 @@ def route_oracle(h_bits: np.ndarray, W_bits: np.ndarray, tau: float,
     return RouteResult(token, conf, entropy, mask, idx, count, gap, tau32)
 
 
+def with_threshold(result: RouteResult, tau: float) -> RouteResult:
+    """The same per-row scores with steps 5-6 redone for another threshold."""
+    mask, idx, count, tau32 = route_decision(result.conf, tau)
+    return RouteResult(result.token, result.conf, result.entropy, mask, idx, count, result.top2_gap, tau32)
+
+
 def percentile_tau(conf: np.ndarray, fraction: float = 0.07) -> float:
     """Threshold that routes exactly the k = max(1, floor(fraction*n)) least confident rows.
 

@@ -1,0 +1,182 @@
+"""ctypes binding of libtlr.so: the same entry points as include/tlr.h, argument marshalling only.
+
+Every step of the routing path runs inside the library's CUDA kernels.  torch is used
+for device memory and streams.  There is no fallback: if the library is missing or a
+call fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from ctypes import POINTER, byref, c_char_p, c_float, c_int32, c_uint32, c_void_p
+
+import torch
+
+PKG_DIR = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(PKG_DIR, "libtlr.so")
+
+TLR_OK = 0
+TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED, TLR_ERR_CUDA = 1, 2, 3, 4
+TLR_ERR_NOMEM, TLR_ERR_TOO_MANY_ROWS, TLR_ERR_DEVICE_STATUS = 5, 6, 7
+TLR_PATH_AUTO, TLR_PATH_SIMT, TLR_PATH_TC = 0, 1, 2
+TLR_DEV_WAIT_TIMEOUT, TLR_DEV_NONFINITE = 1, 2
+
+
+class TlrPlan(ctypes.Structure):
+    _fields_ = [("path", c_int32), ("grid", c_int32), ("block", c_int32), ("row_units", c_int32),
+                ("vocab_chunks", c_int32), ("smem_bytes", c_int32), ("launches", c_int32), ("reserved", c_int32)]
+
+
+class TlrError(RuntimeError):
+    def __init__(self, code: int, where: str):
+        self.code = code
+        super().__init__("%s: %s (status %d)" % (where, status_string(code), code))
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads libtlr.so from the package directory; raises if it has not been built."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise RuntimeError("libtlr.so not found at %s -- build it with `python -m paper_2504_07878_b200.build`"
+                           % LIB_PATH)
+    lib = ctypes.CDLL(LIB_PATH)
+    P = c_void_p
+    lib.tlr_create.argtypes = [c_int32, c_int32, P, c_int32, POINTER(P)]
+    lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_destroy.argtypes = [P]
+    lib.tlr_status_string.argtypes = [c_int32]
+    lib.tlr_status_string.restype = c_char_p
+    lib.tlr_last_device_status.argtypes = [P, POINTER(c_uint32)]
+    lib.tlr_set_path.argtypes = [P, c_int32]
+    lib.tlr_plan_query.argtypes = [P, c_int32, POINTER(TlrPlan)]
+    lib.tlr_set_kernel_timing.argtypes = [P, c_int32]
+    lib.tlr_read_kernel_timing.argtypes = [P, POINTER(c_int32), POINTER(c_float)]
+    for name in ("tlr_create", "tlr_route", "tlr_route_host", "tlr_destroy", "tlr_last_device_status",
+                 "tlr_set_path", "tlr_plan_query", "tlr_set_kernel_timing", "tlr_read_kernel_timing"):
+        getattr(lib, name).restype = c_int32
+    _lib = lib
+    return lib
+
+
+def status_string(code: int) -> str:
+    return load_library().tlr_status_string(code).decode()
+
+
+def _check(code: int, where: str):
+    if code != TLR_OK:
+        raise TlrError(code, where)
+
+
+def _ptr(t) -> c_void_p:
+    if t is None:
+        return c_void_p(0)
+    if isinstance(t, int):
+        return c_void_p(t)
+    return c_void_p(t.data_ptr())
+
+
+def _stream_handle(stream) -> c_void_p:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    if isinstance(stream, int):
+        return c_void_p(stream)
+    return c_void_p(stream.cuda_stream)
+
+
+def tlr_create(d: int, V: int, W, max_n: int) -> c_void_p:
+    """W: CUDA bf16 [V, d] contiguous tensor (or a raw device address).  It is borrowed, not copied."""
+    ctx = c_void_p(0)
+    _check(load_library().tlr_create(d, V, _ptr(W), max_n, byref(ctx)), "tlr_create")
+    return ctx
+
+
+def tlr_route(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count, stream=None):
+    """All tensor arguments are CUDA tensors (or raw device addresses).  Asynchronous on `stream`."""
+    _check(load_library().tlr_route(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy), _ptr(route_mask),
+                                    _ptr(routed_idx), _ptr(routed_count), _stream_handle(stream)), "tlr_route")
+
+
+def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count,
+                   stream=None):
+    """Same with HOST tensors (CPU, ideally pinned); copies in, routes, copies out, synchronises."""
+    _check(load_library().tlr_route_host(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
+                                         _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
+                                         _stream_handle(stream)), "tlr_route_host")
+
+
+def tlr_destroy(ctx):
+    _check(load_library().tlr_destroy(ctx), "tlr_destroy")
+
+
+def tlr_last_device_status(ctx) -> int:
+    out = c_uint32(0)
+    _check(load_library().tlr_last_device_status(ctx, byref(out)), "tlr_last_device_status")
+    return out.value
+
+
+def tlr_set_path(ctx, path: int):
+    _check(load_library().tlr_set_path(ctx, path), "tlr_set_path")
+
+
+def tlr_plan_query(ctx, n: int) -> TlrPlan:
+    plan = TlrPlan()
+    _check(load_library().tlr_plan_query(ctx, n, byref(plan)), "tlr_plan_query")
+    return plan
+
+
+def tlr_set_kernel_timing(ctx, enabled: bool):
+    _check(load_library().tlr_set_kernel_timing(ctx, 1 if enabled else 0), "tlr_set_kernel_timing")
+
+
+def tlr_read_kernel_timing(ctx):
+    n, ms = c_int32(0), c_float(0.0)
+    _check(load_library().tlr_read_kernel_timing(ctx, byref(n), byref(ms)), "tlr_read_kernel_timing")
+    return n.value, ms.value
+
+
+class Router:
+    """Convenience owner of a context and its output tensors (allocation only; no arithmetic)."""
+
+    def __init__(self, W: torch.Tensor, max_n: int):
+        if not (W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.is_contiguous()):
+            raise ValueError("W must be a contiguous CUDA bf16 [V, d] tensor")
+        self.W = W                      # keep the borrowed matrix alive
+        self.V, self.d = W.shape
+        self.max_n = max_n
+        with torch.cuda.device(W.device):
+            self.ctx = tlr_create(self.d, self.V, W, max_n)
+            dev = W.device
+            self.token = torch.empty(max_n, dtype=torch.int32, device=dev)
+            self.conf = torch.empty(max_n, dtype=torch.float32, device=dev)
+            self.entropy = torch.empty(max_n, dtype=torch.float32, device=dev)
+            self.route_mask = torch.empty(max_n, dtype=torch.uint8, device=dev)
+            self.routed_idx = torch.empty(max_n, dtype=torch.int32, device=dev)
+            self.routed_count = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def route(self, h: torch.Tensor, tau: float, stream=None):
+        """Enqueues one routing step; returns views of the output tensors (valid after the stream syncs)."""
+        if not (h.is_cuda and h.dtype == torch.bfloat16 and h.dim() == 2 and h.is_contiguous()
+                and h.shape[1] == self.d):
+            raise ValueError("h must be a contiguous CUDA bf16 [n, d] tensor")
+        n = h.shape[0]
+        tlr_route(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
+                  self.routed_count, stream)
+        return (self.token[:n], self.conf[:n], self.entropy[:n], self.route_mask[:n], self.routed_idx,
+                self.routed_count)
+
+    def close(self):
+        if self.ctx is not None:
+            tlr_destroy(self.ctx)
+            self.ctx = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

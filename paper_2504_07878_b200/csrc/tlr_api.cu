@@ -1,0 +1,383 @@
+// C-ABI of the routing library: context, argument checks, launch planning, dispatch.
+#include <cuda.h>
+#include <cuda_runtime.h>
+
+#include <new>
+#include <vector>
+
+#include "tlr.h"
+#include "tlr_common.cuh"
+#include "tlr_tc.cuh"
+
+namespace tlr {
+
+constexpr int kMaxChunks = 192;       // upper bound on partials per row (sizes the workspace)
+constexpr int kMaxTimedLaunches = 4096;
+
+int tc_choose_chunks(int n, int V, int workers, int max_chunks) {
+  const int row_units = (n + 127) / 128;
+  const int granules = (V + 15) / 16;
+  int hi = granules / 4;               // at least 64 vocabulary rows per chunk
+  if (hi < 1) hi = 1;
+  if (hi > max_chunks) hi = max_chunks;
+  long long best_cost = -1;
+  int best = 1;
+  for (int c = 1; c <= hi; ++c) {
+    const long long rows = 16ll * ((granules + c - 1) / c);
+    const long long units = 1ll * row_units * c;
+    const long long waves = (units + workers - 1) / workers;
+    const long long cost = waves * (rows + 48);
+    if (best_cost < 0 || cost < best_cost) {
+      best_cost = cost;
+      best = c;
+    }
+  }
+  return best;
+}
+
+}  // namespace tlr
+
+using tlr::Partial;
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct tlr_ctx {
+  int device = 0;
+  int sm_count = 0;
+  int d = 0, V = 0, max_n = 0;
+  const void* W = nullptr;
+  tlr_path forced = TLR_PATH_AUTO;
+  bool tc_ok = false;
+  EncodeTiledFn encode = nullptr;
+  CUtensorMap map_w64, map_w16;
+
+  Partial* partials = nullptr;
+  unsigned int* ticket = nullptr;
+  uint32_t* status = nullptr;
+
+  // staging for tlr_route_host
+  void* h_stage = nullptr;
+  int32_t* token_stage = nullptr;
+  float* conf_stage = nullptr;
+  float* entropy_stage = nullptr;
+  uint8_t* mask_stage = nullptr;
+  int32_t* idx_stage = nullptr;
+  int32_t* count_stage = nullptr;
+
+  bool timing = false;
+  std::vector<cudaEvent_t> events;   // pairs, created lazily
+  int timed = 0;
+};
+
+namespace {
+
+bool make_map(tlr_ctx* c, CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols) * 2};
+  const cuuint32_t box[2] = {64u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t elem[2] = {1u, 1u};
+  const CUresult r = c->encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box,
+                               elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+tlr_path pick_path(const tlr_ctx* c) {
+  if (c->forced == TLR_PATH_SIMT) return TLR_PATH_SIMT;
+  return c->tc_ok ? TLR_PATH_TC : TLR_PATH_SIMT;
+}
+
+void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
+  const tlr_path path = pick_path(c);
+  out->path = path;
+  out->launches = n > 0 ? 2 : 1;
+  out->reserved = 0;
+  if (path == TLR_PATH_TC) {
+    const int chunks = tlr::tc_choose_chunks(n, c->V, c->sm_count, tlr::kMaxChunks);
+    const int row_units = (n + 127) / 128;
+    const int units = chunks * row_units;
+    out->vocab_chunks = chunks;
+    out->row_units = row_units;
+    out->grid = units < c->sm_count ? units : c->sm_count;
+    out->block = tlr::tc_threads();
+    out->smem_bytes = tlr::tc_smem_bytes();
+  } else {
+    int chunks, grid, block, smem;
+    tlr::simt_plan(n, c->d, c->V, c->sm_count, &chunks, &grid, &block, &smem);
+    out->vocab_chunks = chunks;
+    out->row_units = (n + 7) / 8;
+    out->grid = grid;
+    out->block = block;
+    out->smem_bytes = smem;
+  }
+}
+
+void free_all(tlr_ctx* c) {
+  cudaFree(c->partials);
+  cudaFree(c->ticket);
+  cudaFree(c->status);
+  cudaFree(c->h_stage);
+  cudaFree(c->token_stage);
+  cudaFree(c->conf_stage);
+  cudaFree(c->entropy_stage);
+  cudaFree(c->mask_stage);
+  cudaFree(c->idx_stage);
+  cudaFree(c->count_stage);
+  for (cudaEvent_t e : c->events) cudaEventDestroy(e);
+  delete c;
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* tlr_status_string(tlr_status s) {
+  switch (s) {
+    case TLR_OK: return "ok";
+    case TLR_ERR_ARG: return "invalid argument";
+    case TLR_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case TLR_ERR_UNSUPPORTED: return "unsupported device or shape";
+    case TLR_ERR_CUDA: return "CUDA call failed";
+    case TLR_ERR_NOMEM: return "device memory allocation failed";
+    case TLR_ERR_TOO_MANY_ROWS: return "n exceeds max_n of the context";
+    case TLR_ERR_DEVICE_STATUS: return "a kernel raised a device status flag";
+  }
+  return "unknown status";
+}
+
+tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_n, tlr_ctx** out) {
+  if (out == nullptr) return TLR_ERR_ARG;
+  *out = nullptr;
+  if (d <= 0 || V <= 0 || max_n <= 0 || W_bf16_dev == nullptr) return TLR_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(W_bf16_dev) & 15u) != 0) return TLR_ERR_ALIGN;
+  if (static_cast<long long>(V) + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TLR_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TLR_ERR_CUDA;
+  if (prop.major != 10) return TLR_ERR_UNSUPPORTED;   // the kernels are built for sm_100a only
+
+  tlr_ctx* c = new (std::nothrow) tlr_ctx();
+  if (c == nullptr) return TLR_ERR_NOMEM;
+  c->device = dev;
+  c->sm_count = prop.multiProcessorCount;
+  c->d = d;
+  c->V = V;
+  c->max_n = max_n;
+  c->W = W_bf16_dev;
+
+  const size_t np = static_cast<size_t>(max_n);
+  bool ok = true;
+  ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->token_stage, np * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->conf_stage, np * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->entropy_stage, np * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->mask_stage, np) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->idx_stage, np * 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->count_stage, 4) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_all(c);
+    return TLR_ERR_NOMEM;
+  }
+  if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
+      cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
+    free_all(c);
+    return TLR_ERR_CUDA;
+  }
+
+  // Tensor-core path: needs 16-byte row pitch for TMA, and the driver's tensor-map encoder.
+  c->tc_ok = false;
+  if (d % 8 == 0) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess && fn != nullptr) {
+      c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+      if (make_map(c, &c->map_w64, W_bf16_dev, V, d, 64) && make_map(c, &c->map_w16, W_bf16_dev, V, d, 16) &&
+          tlr::tc_prepare() == cudaSuccess) {
+        c->tc_ok = true;
+      }
+    }
+    cudaGetLastError();
+    if (!c->tc_ok) {   // on an sm_100 device with d % 8 == 0 this must work; do not fall back silently
+      free_all(c);
+      return TLR_ERR_CUDA;
+    }
+  }
+  *out = c;
+  return TLR_OK;
+}
+
+tlr_status tlr_destroy(tlr_ctx* ctx) {
+  if (ctx == nullptr) return TLR_OK;
+  free_all(ctx);
+  return TLR_OK;
+}
+
+tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path) {
+  if (ctx == nullptr) return TLR_ERR_ARG;
+  if (path != TLR_PATH_AUTO && path != TLR_PATH_SIMT && path != TLR_PATH_TC) return TLR_ERR_ARG;
+  if (path == TLR_PATH_TC && !ctx->tc_ok) return TLR_ERR_UNSUPPORTED;
+  ctx->forced = path;
+  return TLR_OK;
+}
+
+tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out) {
+  if (ctx == nullptr || out == nullptr || n < 0) return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  fill_plan(ctx, n, out);
+  return TLR_OK;
+}
+
+tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, int32_t* token_dev, float* conf_dev,
+                     float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev, int32_t* routed_count_dev,
+                     void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || routed_count_dev == nullptr) return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n > 0) {
+    if (h_bf16_dev == nullptr || token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr ||
+        route_mask_dev == nullptr || routed_idx_dev == nullptr)
+      return TLR_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(h_bf16_dev) & 15u) != 0) return TLR_ERR_ALIGN;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+
+  tlr_plan plan;
+  fill_plan(ctx, n, &plan);
+
+  if (n > 0) {
+    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+    if (ctx->timing && ctx->timed < tlr::kMaxTimedLaunches) {
+      const size_t need = 2 * static_cast<size_t>(ctx->timed + 1);
+      while (ctx->events.size() < need) {
+        cudaEvent_t e;
+        if (cudaEventCreate(&e) != cudaSuccess) return TLR_ERR_CUDA;
+        ctx->events.push_back(e);
+      }
+      ev0 = ctx->events[2 * ctx->timed];
+      ev1 = ctx->events[2 * ctx->timed + 1];
+      if (cudaEventRecord(ev0, stream) != cudaSuccess) return TLR_ERR_CUDA;
+    }
+    cudaError_t e;
+    if (plan.path == TLR_PATH_TC) {
+      CUtensorMap map_h;
+      if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, 128)) return TLR_ERR_CUDA;
+      tlr::TcParams p;
+      p.n = n;
+      p.d = ctx->d;
+      p.V = ctx->V;
+      p.row_units = plan.row_units;
+      p.chunks = plan.vocab_chunks;
+      p.granules = (ctx->V + 15) / 16;
+      p.partials = ctx->partials;
+      p.status = ctx->status;
+      e = tlr::launch_tc_projection(map_h, ctx->map_w64, ctx->map_w16, p, plan.grid, stream);
+    } else {
+      tlr::SimtLaunch a;
+      a.W = ctx->W;
+      a.h = h_bf16_dev;
+      a.n = n;
+      a.d = ctx->d;
+      a.V = ctx->V;
+      a.chunks = plan.vocab_chunks;
+      a.partials = ctx->partials;
+      e = tlr::launch_simt_projection(a, stream);
+    }
+    if (e != cudaSuccess) return TLR_ERR_CUDA;
+    if (ev1 != nullptr) {
+      if (cudaEventRecord(ev1, stream) != cudaSuccess) return TLR_ERR_CUDA;
+      ctx->timed += 1;
+    }
+  }
+
+  tlr::FinishLaunch f;
+  f.partials = ctx->partials;
+  f.n = n;
+  f.chunks = plan.vocab_chunks;
+  f.tau = tau;
+  f.token = token_dev;
+  f.conf = conf_dev;
+  f.entropy = entropy_dev;
+  f.route_mask = route_mask_dev;
+  f.routed_idx = routed_idx_dev;
+  f.routed_count = routed_count_dev;
+  f.ticket = ctx->ticket;
+  f.status = ctx->status;
+  if (tlr::launch_finish(f, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau, int32_t* token_host,
+                          float* conf_host, float* entropy_host, uint8_t* route_mask_host, int32_t* routed_idx_host,
+                          int32_t* routed_count_host, void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || routed_count_host == nullptr) return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n > 0 && h_bf16_host == nullptr) return TLR_ERR_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const size_t nn = static_cast<size_t>(n);
+  if (n > 0 &&
+      cudaMemcpyAsync(ctx->h_stage, h_bf16_host, nn * ctx->d * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return TLR_ERR_CUDA;
+  const tlr_status st = tlr_route(ctx, ctx->h_stage, n, tau, ctx->token_stage, ctx->conf_stage, ctx->entropy_stage,
+                                  ctx->mask_stage, ctx->idx_stage, ctx->count_stage, cuda_stream);
+  if (st != TLR_OK) return st;
+  bool ok = true;
+  if (n > 0) {
+    if (token_host) ok = ok && cudaMemcpyAsync(token_host, ctx->token_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (conf_host) ok = ok && cudaMemcpyAsync(conf_host, ctx->conf_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (entropy_host) ok = ok && cudaMemcpyAsync(entropy_host, ctx->entropy_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (route_mask_host) ok = ok && cudaMemcpyAsync(route_mask_host, ctx->mask_stage, nn, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  }
+  uint32_t dev_status = 0;
+  ok = ok && cudaMemcpyAsync(routed_count_host, ctx->count_stage, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaMemcpyAsync(&dev_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+  if (!ok) return TLR_ERR_CUDA;
+  const int32_t count = *routed_count_host;
+  if (routed_idx_host != nullptr && count > 0) {
+    if (cudaMemcpyAsync(routed_idx_host, ctx->idx_stage, static_cast<size_t>(count) * 4, cudaMemcpyDeviceToHost,
+                        stream) != cudaSuccess ||
+        cudaStreamSynchronize(stream) != cudaSuccess)
+      return TLR_ERR_CUDA;
+  }
+  if (dev_status & TLR_DEV_WAIT_TIMEOUT) return TLR_ERR_DEVICE_STATUS;
+  return TLR_OK;
+}
+
+tlr_status tlr_last_device_status(tlr_ctx* ctx, uint32_t* out_host) {
+  if (ctx == nullptr || out_host == nullptr) return TLR_ERR_ARG;
+  if (cudaDeviceSynchronize() != cudaSuccess) return TLR_ERR_CUDA;
+  if (cudaMemcpy(out_host, ctx->status, 4, cudaMemcpyDeviceToHost) != cudaSuccess) return TLR_ERR_CUDA;
+  if (cudaMemset(ctx->status, 0, 4) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_set_kernel_timing(tlr_ctx* ctx, int32_t enabled) {
+  if (ctx == nullptr) return TLR_ERR_ARG;
+  ctx->timing = enabled != 0;
+  return TLR_OK;
+}
+
+tlr_status tlr_read_kernel_timing(tlr_ctx* ctx, int32_t* launches_out, float* total_ms_out) {
+  if (ctx == nullptr || launches_out == nullptr || total_ms_out == nullptr) return TLR_ERR_ARG;
+  float total = 0.f;
+  for (int i = 0; i < ctx->timed; ++i) {
+    if (cudaEventSynchronize(ctx->events[2 * i + 1]) != cudaSuccess) return TLR_ERR_CUDA;
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, ctx->events[2 * i], ctx->events[2 * i + 1]) != cudaSuccess) return TLR_ERR_CUDA;
+    total += ms;
+  }
+  *launches_out = ctx->timed;
+  *total_ms_out = total;
+  ctx->timed = 0;
+  return TLR_OK;
+}
+
+}  // extern "C"

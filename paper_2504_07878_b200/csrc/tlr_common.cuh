@@ -1,0 +1,105 @@
+// Shared device-side definitions of the routing kernels: the per-row partial result
+// that the projection kernels emit and the rule that merges two of them.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tlr.h"
+
+namespace tlr {
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+constexpr int kNoToken = 0x7fffffff;
+
+// Online-softmax summary of one row over a range of the vocabulary:
+//   m   = max logit in the range          idx = lowest vocabulary index attaining it
+//   s   = sum exp(z - m)                  t   = sum exp(z - m) * (z - m)
+// With the whole vocabulary folded in: conf = 1/s, entropy = ln s - t/s.
+// An empty range is (m = -inf, idx = kNoToken, s = 0, t = 0).
+struct __align__(16) Partial {
+  float m;
+  int idx;
+  float s;
+  float t;
+};
+
+__device__ __forceinline__ Partial empty_partial() {
+  Partial p;
+  p.m = -INFINITY;
+  p.idx = kNoToken;
+  p.s = 0.f;
+  p.t = 0.f;
+  return p;
+}
+
+// Associative and commutative merge; ties on m go to the lower vocabulary index.
+__device__ __forceinline__ Partial merge(const Partial& a, const Partial& b) {
+  Partial r;
+  const bool a_wins = (a.m > b.m) || (a.m == b.m && a.idx <= b.idx);
+  r.m = a_wins ? a.m : b.m;
+  r.idx = a_wins ? a.idx : b.idx;
+  // Rescale each side to the new maximum.  A side with s == 0 contributes nothing
+  // (its m may be -inf, which must not reach the arithmetic below).
+  float s = 0.f, t = 0.f;
+  if (a.s > 0.f) {
+    const float da = a.m - r.m;  // <= 0
+    const float ea = exp2f(da * kLog2e);
+    s += a.s * ea;
+    t += ea * (a.t + da * a.s);
+  }
+  if (b.s > 0.f) {
+    const float db = b.m - r.m;
+    const float eb = exp2f(db * kLog2e);
+    s += b.s * eb;
+    t += eb * (b.t + db * b.s);
+  }
+  r.s = s;
+  r.t = t;
+  return r;
+}
+
+__device__ __forceinline__ Partial shfl_xor(const Partial& p, int lane_mask) {
+  Partial r;
+  r.m = __shfl_xor_sync(0xffffffffu, p.m, lane_mask);
+  r.idx = __shfl_xor_sync(0xffffffffu, p.idx, lane_mask);
+  r.s = __shfl_xor_sync(0xffffffffu, p.s, lane_mask);
+  r.t = __shfl_xor_sync(0xffffffffu, p.t, lane_mask);
+  return r;
+}
+
+__device__ __forceinline__ Partial warp_merge(Partial p) {
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) p = merge(p, shfl_xor(p, off));
+  return p;
+}
+
+// Host-side launchers (one per .cu file).  All enqueue on `stream` and return the
+// launch error, if any.
+struct SimtLaunch {
+  const void* W;
+  const void* h;
+  int n, d, V;
+  int chunks;       // vocabulary chunks (partials per row)
+  Partial* partials;  // [n][chunks]
+};
+cudaError_t launch_simt_projection(const SimtLaunch& a, cudaStream_t stream);
+void simt_plan(int n, int d, int V, int sm_count, int* chunks, int* grid, int* block, int* smem);
+
+struct FinishLaunch {
+  const Partial* partials;  // [n][chunks]
+  int n, chunks;
+  float tau;
+  int32_t* token;
+  float* conf;
+  float* entropy;
+  uint8_t* route_mask;
+  int32_t* routed_idx;
+  int32_t* routed_count;
+  unsigned int* ticket;     // zero before the launch; the kernel leaves it zero again
+  uint32_t* status;
+};
+cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
+
+}  // namespace tlr

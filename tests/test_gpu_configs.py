@@ -1,0 +1,110 @@
+"""GPU parity at the full benchmark sizes, in the launch configuration the benchmark times."""
+import numpy as np
+import pytest
+import torch
+
+import tlr_synth as S
+from oracle import route_oracle as O
+from tests.parity import check_against_oracle, check_self_consistency, run_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+class Head:
+    """W on the host (bits + fp64) and on the device, built once per (d, V)."""
+    _cache = {}
+
+    @classmethod
+    def get(cls, d, V):
+        key = (d, V)
+        if key not in cls._cache:
+            cls._cache.clear()                      # one head at a time: the fp64 copy is 1-2 GB
+            W = S.make_W(d, V, seed=0)
+            cls._cache[key] = (W, O.bf16_bits_to_f64(S.bf16_bits(W)), W.cuda())
+        return cls._cache[key]
+
+
+def oracle_rows(hid, W, W64, tau, rows=None):
+    hb = S.bf16_bits(hid.h)
+    if rows is not None:
+        hb = hb[rows]
+    return O.route_oracle(hb, S.bf16_bits(W), tau, W64=W64)
+
+
+def test_config_decode16_percentile_tau(pkg):
+    wl = S.WORKLOADS["decode16"]
+    W, W64, Wd = Head.get(wl.d, wl.V)
+    hid = S.make_h(wl.n, wl.d, seed=0)
+    first = oracle_rows(hid, W, W64, 0.5)
+    tau = O.percentile_tau(first.conf, 0.07)
+    ref = O.with_threshold(first, tau)
+    assert ref.routed_count == 1
+    gpu = run_gpu(pkg, Wd, hid.h, tau)
+    assert gpu["status"] == 0 and gpu["plan"].path == 2
+    check_self_consistency(gpu, tau, wl.V)
+    rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64)
+    assert rep["route_exempt_rows"] == 0
+    assert gpu["routed_count"] == 1 and gpu["routed_idx"][0] == ref.routed_idx[0]
+
+
+def test_config_decode256(pkg):
+    wl = S.WORKLOADS["decode256"]
+    W, W64, Wd = Head.get(wl.d, wl.V)
+    hid = S.make_h(wl.n, wl.d, seed=0)
+    ref = oracle_rows(hid, W, W64, wl.tau)
+    gpu = run_gpu(pkg, Wd, hid.h, wl.tau)
+    assert gpu["status"] == 0 and gpu["plan"].path == 2
+    check_self_consistency(gpu, wl.tau, wl.V)
+    check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64)
+    assert gpu["routed_count"] == 256 and np.array_equal(gpu["routed_idx"], np.arange(256))
+
+
+def test_config_prefill8192_planted(pkg):
+    wl = S.WORKLOADS["prefill8192"]
+    W, W64, Wd = Head.get(wl.d, wl.V)
+    hid = S.make_h(wl.n, wl.d, seed=0, W=W, planted_fraction=wl.planted_fraction)
+    gpu = run_gpu(pkg, Wd, hid.h, wl.tau)
+    assert gpu["status"] == 0 and gpu["plan"].path == 2
+    check_self_consistency(gpu, wl.tau, wl.V)
+    # every planted row and a seeded sample of the others, computed one by one by the oracle
+    rng = np.random.default_rng(0)
+    others = np.setdiff1d(np.arange(wl.n), hid.planted_rows)
+    rows = np.sort(np.concatenate([hid.planted_rows, rng.choice(others, 1024, replace=False)]))
+    ref = oracle_rows(hid, W, W64, wl.tau, rows)
+    check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64, rows=rows)
+    # planted rows keep the small model's token; everything else is routed: 8192 - 409 = 7783
+    assert np.array_equal(gpu["token"][hid.planted_rows], hid.planted_tokens)
+    assert gpu["routed_count"] == wl.n - hid.planted_rows.size == 7783
+    assert np.array_equal(gpu["routed_idx"][:7783], others.astype(np.int32))
+
+
+def test_config_head1p5b_percentile_tau(pkg):
+    wl = S.WORKLOADS["head1p5b"]
+    W, W64, Wd = Head.get(wl.d, wl.V)
+    hid = S.make_h(wl.n, wl.d, seed=0)
+    first = oracle_rows(hid, W, W64, 0.5)                    # all 4096 rows: tau needs every confidence
+    tau = O.percentile_tau(first.conf, 0.07)
+    ref = O.with_threshold(first, tau)
+    assert ref.routed_count == 286
+    gpu = run_gpu(pkg, Wd, hid.h, tau)
+    assert gpu["status"] == 0 and gpu["plan"].path == 2
+    check_self_consistency(gpu, tau, wl.V)
+    rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64)
+    if rep["route_exempt_rows"] == 0:
+        assert gpu["routed_count"] == 286 and np.array_equal(gpu["routed_idx"][:286], ref.routed_idx)
+
+
+@pytest.mark.parametrize("n", S.SWEEP_N)
+def test_config_sweep(pkg, n):
+    wl = S.WORKLOADS["sweep%d" % n]
+    W, W64, Wd = Head.get(wl.d, wl.V)
+    hid = S.make_h(n, wl.d, seed=0)
+    rows = None if n <= 512 else np.sort(np.random.default_rng(n).choice(n, 256, replace=False))
+    for tau in S.SWEEP_TAU:
+        gpu = run_gpu(pkg, Wd, hid.h, tau, max_n=n)
+        assert gpu["status"] == 0 and gpu["plan"].path == 2
+        check_self_consistency(gpu, tau, wl.V)
+        assert gpu["routed_count"] == n and np.array_equal(gpu["routed_idx"], np.arange(n))   # conf ~1e-4 << tau
+        if tau == S.SWEEP_TAU[0]:
+            ref = oracle_rows(hid, W, W64, tau, rows)
+            check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64, rows=rows)
