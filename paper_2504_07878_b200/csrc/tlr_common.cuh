@@ -40,16 +40,17 @@ __device__ __forceinline__ Partial merge(const Partial& a, const Partial& b) {
   const bool a_wins = (a.m > b.m) || (a.m == b.m && a.idx <= b.idx);
   r.m = a_wins ? a.m : b.m;
   r.idx = a_wins ? a.idx : b.idx;
-  // Rescale each side to the new maximum.  A side with s == 0 contributes nothing
-  // (its m may be -inf, which must not reach the arithmetic below).
+  // Rescale each side to the new maximum.  A side with s == 0 (an empty range) contributes
+  // nothing: its m is -inf, which must not reach the arithmetic below.  A NaN sum is not
+  // "empty": it goes through and poisons the result, which the final step then flags.
   float s = 0.f, t = 0.f;
-  if (a.s > 0.f) {
+  if (!(a.s == 0.f)) {
     const float da = a.m - r.m;  // <= 0
     const float ea = exp2f(da * kLog2e);
     s += a.s * ea;
     t += ea * (a.t + da * a.s);
   }
-  if (b.s > 0.f) {
+  if (!(b.s == 0.f)) {
     const float db = b.m - r.m;
     const float eb = exp2f(db * kLog2e);
     s += b.s * eb;

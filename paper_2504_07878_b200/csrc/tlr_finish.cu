@@ -42,6 +42,8 @@ finish_kernel(const FinishLaunch a) {
         conf = fminf(conf, 1.0f);
         ent = fmaxf(ent, 0.0f);
       } else {
+        conf = __int_as_float(0x7fc00000);   // NaN: fails "conf >= tau", so the row is routed
+        ent = conf;
         atomicOr(a.status, TLR_DEV_NONFINITE);
       }
       a.token[row] = acc.idx;

@@ -15,7 +15,7 @@
 //   warp 1   MMA issuer: one thread issues tcgen05.mma (M=128, N=tile, K=16) x4 per slab
 //            into one of two 256-column TMEM accumulators; also owns TMEM alloc/free
 //   warps 2-5 epilogue: each owns 32 TMEM lanes (rows); reads the finished accumulator
-//            32 columns at a time and folds it into per-row (m, idx, s, u) registers
+//            32 columns at a time and folds it into per-row (m, idx, S, T) registers
 //            while the next tile's MMAs run into the other accumulator.
 // At the end of a unit every row's summary is written as one 16-byte partial.
 //
@@ -334,13 +334,17 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
       const UnitRange u = unit_range(p, unit);
       const int chunk = unit / p.row_units;
       const int G = u.g1 - u.g0;
-      const int T = (G * 16 + kBlockN - 1) / kBlockN;
+      const int T_tiles = (G * 16 + kBlockN - 1) / kBlockN;
       const bool warp_has_rows = (u.row0 + quad * 32) < p.n;   // warp-uniform
-      float m = -INFINITY, s0 = 0.f, s1 = 0.f, u0 = 0.f, u1 = 0.f;
+      // Running summary of this thread's row over the unit.  S = sum 2^y and T = sum 2^y * y
+      // with y = (z - m) * log2(e) <= 0; both are accumulated per 32-column group first and
+      // then added with a compensated (Kahan) sum, so that one dominant term -- a confident
+      // row has S ~ 1 with thousands of terms ~1e-8 after it -- does not swallow the rest.
+      float m = -INFINITY, S = 0.f, cS = 0.f, T = 0.f, cT = 0.f;
       int idx = kNoToken;
-      for (int t = 0; t < T && ok; ++t) {
+      for (int t = 0; t < T_tiles && ok; ++t) {
         int ga, gb;
-        tile_range(G, T, t, &ga, &gb);
+        tile_range(G, T_tiles, t, &ga, &gb);
         const int v0 = (u.g0 + ga) * 16;
         const int cols = min((gb - ga) * 16, p.V - v0);   // valid columns of this tile
         if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
@@ -356,15 +360,19 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
             if (valid < 32) {
 #pragma unroll
               for (int j = 0; j < 32; ++j)
-                if (j >= valid) z[j] = -1.0e30f;   // finite, so 0 * z stays 0 below
+                if (j >= valid) z[j] = -1.0e30f;   // finite, so 0 * y stays 0 below
             }
             float cm = z[0];
 #pragma unroll
             for (int j = 1; j < 32; ++j) cm = fmaxf(cm, z[j]);
             if (cm > m) {
               if (m != -INFINITY) {
-                const float sc = ex2_approx((m - cm) * kLog2e);
-                s0 *= sc; s1 *= sc; u0 *= sc; u1 *= sc;
+                const float dl = (cm - m) * kLog2e;       // > 0
+                const float sc = ex2_approx(-dl);
+                T = sc * (T - dl * S);
+                cT *= sc;
+                S *= sc;
+                cS *= sc;
               }
               m = cm;
               int first = 31;
@@ -373,14 +381,29 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
               idx = v0 + c0 + first;
             }
             const float neg_ml = -m * kLog2e;
+            float ls0 = 0.f, ls1 = 0.f, lt0 = 0.f, lt1 = 0.f;
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-              const float e0 = ex2_approx(fmaf(z[j], kLog2e, neg_ml));
-              const float e1 = ex2_approx(fmaf(z[j + 1], kLog2e, neg_ml));
-              s0 += e0;
-              s1 += e1;
-              u0 = fmaf(e0, z[j], u0);
-              u1 = fmaf(e1, z[j + 1], u1);
+              const float y0 = fmaf(z[j], kLog2e, neg_ml);
+              const float y1 = fmaf(z[j + 1], kLog2e, neg_ml);
+              const float e0 = ex2_approx(y0);
+              const float e1 = ex2_approx(y1);
+              ls0 += e0;
+              ls1 += e1;
+              lt0 = fmaf(e0, y0, lt0);
+              lt1 = fmaf(e1, y1, lt1);
+            }
+            {
+              const float a = (ls0 + ls1) - cS;
+              const float b = S + a;
+              cS = (b - S) - a;
+              S = b;
+            }
+            {
+              const float a = (lt0 + lt1) - cT;
+              const float b = T + a;
+              cT = (b - T) - a;
+              T = b;
             }
           }
         }
@@ -390,12 +413,11 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
       if (ok && u.row0 + row_in_unit < p.n) {
-        const float s = s0 + s1;
         Partial out;
         out.m = m;
         out.idx = idx;
-        out.s = s;
-        out.t = (u0 + u1) - m * s;     // sum e^(z-m) (z-m)
+        out.s = S;
+        out.t = T * kLn2;              // sum e^(z-m) (z-m), back in nats
         p.partials[static_cast<size_t>(u.row0 + row_in_unit) * p.chunks + chunk] = out;
       }
     }
