@@ -158,6 +158,42 @@ tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out);
 tlr_status tlr_set_kernel_timing(tlr_ctx* ctx, int32_t enabled);
 tlr_status tlr_read_kernel_timing(tlr_ctx* ctx, int32_t* launches_out, float* total_ms_out);
 
+/*
+ * tlr_route_static -- the routing step for callers that cannot allocate device memory.
+ * (No counterpart in the paper: this is a deployment convenience of the library.)
+ *
+ * Who needs it: a serving process that has already given all free HBM to its own pools,
+ * so that a cudaMalloc would fail or disturb them; a decode loop that cannot tolerate the
+ * device-wide synchronisation an allocation may cause; a plug-in whose host forbids
+ * allocation in its callbacks.  tlr_create allocates a workspace, so such callers cannot
+ * use it; this call needs no context and calls no cudaMalloc, cudaFree or other
+ * allocating routine.  Its scratch (per-row partial results and a ticket counter) is a
+ * fixed array inside the library image, about 3 MiB, which every GPU that loads the
+ * library holds until the process exits.
+ *
+ * Arguments are those of tlr_create + tlr_route: d, V and W (bf16 [V,d], 16-byte aligned,
+ * only read), then h, n, tau and the six outputs with the same layouts and meaning.
+ *   n           0 <= n <= TLR_STATIC_MAX_ROWS; more rows return TLR_ERR_TOO_MANY_ROWS
+ *               (the fixed scratch cannot hold them; use a context for larger batches).
+ *   status_dev  optional uint32 [1] on the device: receives the TLR_DEV_* flags of this
+ *               call (cleared at its start).  NULL keeps the flags in the scratch, unread.
+ * Asynchronous on cuda_stream like tlr_route.
+ *
+ * The first call on each device performs a one-time set-up for that device (it looks up
+ * the scratch array's device address and opts the kernels in to their shared-memory
+ * size); make that first call outside any stream capture.  All calls share the one
+ * scratch array, which keeps the previous call's contents (the call clears what must
+ * start at zero): calls must not overlap on the GPU -- issue them on one stream, or
+ * order them yourself; two calls in flight at once race.
+ * Errors: TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_TOO_MANY_ROWS, TLR_ERR_UNSUPPORTED (device
+ * is not sm_100), TLR_ERR_CUDA.
+ */
+#define TLR_STATIC_MAX_ROWS 1024
+tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_dev, const void* h_bf16_dev,
+                            int32_t n, float tau, int32_t* token_dev, float* conf_dev,
+                            float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev,
+                            int32_t* routed_count_dev, uint32_t* status_dev, void* cuda_stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -20,6 +20,7 @@ TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED, TLR_ERR_CUDA = 1, 2, 3, 4
 TLR_ERR_NOMEM, TLR_ERR_TOO_MANY_ROWS, TLR_ERR_DEVICE_STATUS = 5, 6, 7
 TLR_PATH_AUTO, TLR_PATH_SIMT, TLR_PATH_TC = 0, 1, 2
 TLR_DEV_WAIT_TIMEOUT, TLR_DEV_NONFINITE = 1, 2
+TLR_STATIC_MAX_ROWS = 1024
 
 
 class TlrPlan(ctypes.Structure):
@@ -57,6 +58,8 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_plan_query.argtypes = [P, c_int32, POINTER(TlrPlan)]
     lib.tlr_set_kernel_timing.argtypes = [P, c_int32]
     lib.tlr_read_kernel_timing.argtypes = [P, POINTER(c_int32), POINTER(c_float)]
+    lib.tlr_route_static.argtypes = [c_int32, c_int32, P, P, c_int32, c_float, P, P, P, P, P, P, P, P]
+    lib.tlr_route_static.restype = c_int32
     for name in ("tlr_create", "tlr_route", "tlr_route_host", "tlr_destroy", "tlr_last_device_status",
                  "tlr_set_path", "tlr_plan_query", "tlr_set_kernel_timing", "tlr_read_kernel_timing"):
         getattr(lib, name).restype = c_int32
@@ -108,6 +111,19 @@ def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask,
     _check(load_library().tlr_route_host(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
                                          _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
                                          _stream_handle(stream)), "tlr_route_host")
+
+
+def tlr_route_static(d: int, V: int, W, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx,
+                     routed_count, status=None, stream=None):
+    """The routing step without a context and without any device allocation (at most TLR_STATIC_MAX_ROWS rows).
+
+    For callers that may not allocate GPU memory; the scratch is a fixed array inside the library,
+    shared by all calls, so calls must not overlap on the GPU.  Make the first call on a device
+    outside stream capture (it does a one-time set-up).
+    """
+    _check(load_library().tlr_route_static(d, V, _ptr(W), _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
+                                           _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count), _ptr(status),
+                                           _stream_handle(stream)), "tlr_route_static")
 
 
 def tlr_destroy(ctx):
