@@ -14,25 +14,34 @@ namespace tlr {
 constexpr int kMaxChunks = 192;       // upper bound on partials per row (sizes the workspace)
 constexpr int kMaxTimedLaunches = 4096;
 
-int tc_choose_chunks(int n, int V, int workers, int max_chunks) {
-  const int row_units = (n + 127) / 128;
-  const int granules = (V + 15) / 16;
-  int hi = granules / 4;               // at least 64 vocabulary rows per chunk
+// Chooses the vocabulary decomposition: every unit gets the same number of tiles, and the
+// number of chunks minimises (waves of units) x (rows of the largest chunk + a fixed cost
+// per tile), so that workers finish together.
+void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
+  const int g = 16 * cta;
+  const int row_units = (n + 128 * cta - 1) / (128 * cta);
+  const int granules = (V + g - 1) / g;
+  int hi = granules < max_chunks ? granules : max_chunks;
   if (hi < 1) hi = 1;
-  if (hi > max_chunks) hi = max_chunks;
   long long best_cost = -1;
-  int best = 1;
+  int best = 1, best_tiles = 1;
   for (int c = 1; c <= hi; ++c) {
-    const long long rows = 16ll * ((granules + c - 1) / c);
+    const long long gmax = (granules + c - 1) / c;
+    const long long tiles = (gmax * g + 255) / 256;
     const long long units = 1ll * row_units * c;
     const long long waves = (units + workers - 1) / workers;
-    const long long cost = waves * (rows + 48);
+    const long long cost = waves * (gmax * g + 24 * tiles);
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = c;
+      best_tiles = static_cast<int>(tiles);
     }
   }
-  return best;
+  plan->row_units = row_units;
+  plan->chunks = best;
+  plan->granule_rows = g;
+  plan->granules = granules;
+  plan->tiles_per_unit = best_tiles;
 }
 
 }  // namespace tlr
@@ -95,14 +104,18 @@ void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
   out->launches = n > 0 ? 2 : 1;
   out->reserved = 0;
   if (path == TLR_PATH_TC) {
-    const int chunks = tlr::tc_choose_chunks(n, c->V, c->sm_count, tlr::kMaxChunks);
-    const int row_units = (n + 127) / 128;
-    const int units = chunks * row_units;
-    out->vocab_chunks = chunks;
-    out->row_units = row_units;
-    out->grid = units < c->sm_count ? units : c->sm_count;
+    tlr::TcConfig cfg;
+    tlr::TcPlan tp;
+    tlr::tc_configure(n, &cfg);
+    const int workers_max = c->sm_count / cfg.cta;
+    tlr::tc_plan(n, c->V, cfg.cta, workers_max, tlr::kMaxChunks, &tp);
+    const int units = tp.chunks * tp.row_units;
+    const int workers = units < workers_max ? units : workers_max;
+    out->vocab_chunks = tp.chunks;
+    out->row_units = tp.row_units;
+    out->grid = workers * cfg.cta;
     out->block = tlr::tc_threads();
-    out->smem_bytes = tlr::tc_smem_bytes();
+    out->smem_bytes = cfg.smem_bytes;
   } else {
     int chunks, grid, block, smem;
     tlr::simt_plan(n, c->d, c->V, c->sm_count, &chunks, &grid, &block, &smem);
@@ -267,18 +280,26 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
     }
     cudaError_t e;
     if (plan.path == TLR_PATH_TC) {
+      tlr::TcConfig cfg;
+      tlr::TcPlan tp;
+      tlr::tc_configure(n, &cfg);
+      tlr::tc_plan(n, ctx->V, cfg.cta, ctx->sm_count / cfg.cta, tlr::kMaxChunks, &tp);
       CUtensorMap map_h;
-      if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, 128)) return TLR_ERR_CUDA;
+      if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
       tlr::TcParams p;
       p.n = n;
       p.d = ctx->d;
       p.V = ctx->V;
-      p.row_units = plan.row_units;
-      p.chunks = plan.vocab_chunks;
-      p.granules = (ctx->V + 15) / 16;
+      p.row_units = tp.row_units;
+      p.chunks = tp.chunks;
+      p.granules = tp.granules;
+      p.tiles_per_unit = tp.tiles_per_unit;
+      p.a_rows = cfg.a_rows;
+      p.a_stages = cfg.a_stages;
+      p.b_stages = cfg.b_stages;
       p.partials = ctx->partials;
       p.status = ctx->status;
-      e = tlr::launch_tc_projection(map_h, ctx->map_w64, ctx->map_w16, p, plan.grid, stream);
+      e = tlr::launch_tc_projection(map_h, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
     } else {
       tlr::SimtLaunch a;
       a.W = ctx->W;

@@ -128,24 +128,32 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
   if (n > 0) {
     if (d % 8 == 0 && !s->tc_ready) return TLR_ERR_CUDA;   // no silent change of kernel
     if (d % 8 == 0) {
-      chunks = tlr::tc_choose_chunks(n, V, s->sm_count, kStaticMaxChunks);
-      const int row_units = (n + 127) / 128;
-      const int units = chunks * row_units;
+      tlr::TcConfig cfg;
+      tlr::TcPlan tp;
+      tlr::tc_configure(n, &cfg);
+      const int workers_max = s->sm_count / cfg.cta;
+      tlr::tc_plan(n, V, cfg.cta, workers_max, kStaticMaxChunks, &tp);
+      chunks = tp.chunks;
+      const int units = tp.chunks * tp.row_units;
       CUtensorMap map_h, map_w64, map_w16;
-      if (!encode_map(&map_h, h_bf16_dev, n, d, 128) || !encode_map(&map_w64, W_bf16_dev, V, d, 64) ||
+      if (!encode_map(&map_h, h_bf16_dev, n, d, cfg.a_rows) || !encode_map(&map_w64, W_bf16_dev, V, d, 64) ||
           !encode_map(&map_w16, W_bf16_dev, V, d, 16))
         return TLR_ERR_CUDA;
       tlr::TcParams p;
       p.n = n;
       p.d = d;
       p.V = V;
-      p.row_units = row_units;
-      p.chunks = chunks;
-      p.granules = (V + 15) / 16;
+      p.row_units = tp.row_units;
+      p.chunks = tp.chunks;
+      p.granules = tp.granules;
+      p.tiles_per_unit = tp.tiles_per_unit;
+      p.a_rows = cfg.a_rows;
+      p.a_stages = cfg.a_stages;
+      p.b_stages = cfg.b_stages;
       p.partials = partials;
       p.status = status;
-      if (tlr::launch_tc_projection(map_h, map_w64, map_w16, p, units < s->sm_count ? units : s->sm_count, stream) !=
-          cudaSuccess)
+      if (tlr::launch_tc_projection(map_h, map_w64, map_w16, p, cfg, units < workers_max ? units : workers_max,
+                                    stream) != cudaSuccess)
         return TLR_ERR_CUDA;
     } else {
       int grid, block, smem;

@@ -3,24 +3,38 @@
 // online-softmax reduction (max / argmax / sum-exp / entropy numerator) fused into
 // the epilogue, so the n x V logits never leave the SM.
 //
-// Decomposition.  The vocabulary is cut into `chunks` contiguous ranges of 16-row
-// granules; the token rows into units of 128 (one TMEM lane per row).  A work unit is
-// (chunk, row unit); units are numbered chunk-major so that CTAs running at the same
-// time share W tiles through L2, and each persistent CTA takes units blockIdx.x,
-// blockIdx.x + gridDim.x, ...  Inside a unit the chunk is walked in tiles of at most
-// 256 vocabulary rows (the MMA's N), each a K-loop over d in slabs of 64 elements.
+// Two instantiations of one kernel:
+//   kCta = 1  one CTA per worker, MMA M = 128 token rows            (n <= 128)
+//   kCta = 2  a cluster of two CTAs per worker, MMA M = 256 rows (cta_group::2): each
+//             CTA stages its own 128 rows of h and HALF of the W tile, and the pair's
+//             tensor cores read both halves, so a W byte enters shared memory once
+//             per 256 token rows.                                   (n > 128)
 //
-// Roles (warp-specialised, 192 threads):
-//   warp 0   TMA producer: fills a ring of kStages {h slab 128x64, W slab Nx64} buffers
-//   warp 1   MMA issuer: one thread issues tcgen05.mma (M=128, N=tile, K=16) x4 per slab
-//            into one of two 256-column TMEM accumulators; also owns TMEM alloc/free
+// Decomposition.  The vocabulary is cut into `chunks` contiguous ranges of granules
+// (16 * kCta rows); the token rows into units of 128 * kCta.  A work unit is
+// (chunk, row unit); units are numbered chunk-major so that workers running at the
+// same time share W through L2, and worker w takes units w, w + workers, ...  Inside
+// a unit the chunk is walked in `tiles_per_unit` tiles of at most 256 vocabulary rows
+// (the MMA's N), each a K-loop over d in slabs of 64 elements.
+//
+// Roles (warp-specialised, 224 threads per CTA):
+//   warp 0   W producer: TMA loads of W slabs into a deep ring (W comes from HBM)
+//   warp 6   h producer: TMA loads of h slabs into a short ring (h comes from L2)
+//   warp 1   MMA issuer (leader CTA only): tcgen05.mma x4 per slab into one of two
+//            256-column TMEM accumulators; also owns TMEM alloc/free
 //   warps 2-5 epilogue: each owns 32 TMEM lanes (rows); reads the finished accumulator
 //            32 columns at a time and folds it into per-row (m, idx, S, T) registers
 //            while the next tile's MMAs run into the other accumulator.
 // At the end of a unit every row's summary is written as one 16-byte partial.
 //
+// How much of W a CTA keeps in flight decides its streaming rate (latency-bound
+// otherwise), so h slabs get their own small ring and, when n is small, a slab of only
+// as many rows as n needs; the MMA then reads its remaining A rows from whatever
+// follows in shared memory, which only affects accumulator rows that are never used.
+//
 // Every mbarrier wait is bounded (wall-clock limit); on expiry the kernel raises
-// TLR_DEV_WAIT_TIMEOUT, drains its outstanding copies, frees TMEM and returns.
+// TLR_DEV_WAIT_TIMEOUT, lets its outstanding copies land, frees TMEM and returns.
+// No TMA load uses cluster multicast.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -31,20 +45,20 @@ namespace tlr {
 
 namespace {
 
-constexpr int kBlockM = 128;                 // token rows per unit == TMEM lanes
+constexpr int kBlockM = 128;                 // token rows per CTA == TMEM lanes
 constexpr int kBlockN = 256;                 // max vocabulary rows per tile == accumulator columns
 constexpr int kBlockK = 64;                  // bf16 per slab row = 128 B = one swizzle span
 constexpr int kUmmaK = 16;
-constexpr int kStages = 4;
-constexpr int kABytes = kBlockM * kBlockK * 2;   // 16 KiB
-constexpr int kBBytes = kBlockN * kBlockK * 2;   // 32 KiB
-constexpr int kStageBytes = kABytes + kBBytes;
+constexpr int kRowBytes = kBlockK * 2;       // 128
 constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 4;
-constexpr int kThreads = 32 * (2 + kEpiWarps);
-constexpr int kBarrierBytes = 256;
-constexpr int kSmemBytes = 1024 + kStages * kStageBytes + kBarrierBytes;
+constexpr int kThreads = 32 * 7;
+constexpr int kMaxAStages = 4;
+constexpr int kMaxBStages = 12;
+constexpr int kBarrierBytes = 512;
+constexpr int kSmemLimit = 232448;           // 227 KiB opt-in maximum per CTA
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
+constexpr unsigned long long kDrainNs = 200000ull;          // 200 us: far beyond any copy's flight time
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -56,6 +70,22 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 
+__device__ __forceinline__ uint32_t cluster_ctarank() {
+  uint32_t r;
+  asm volatile("mov.u32 %0, %cluster_ctarank;" : "=r"(r));
+  return r;
+}
+// Address of the same shared-memory offset in CTA `rank` of this cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
 }
@@ -64,6 +94,10 @@ __device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
 }
 __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+// Arrive on a barrier given by a shared::cluster address (own CTA or the peer).
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
 }
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   uint32_t ok;
@@ -95,38 +129,90 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
   }
 }
 
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
-      : "memory");
+// After giving up: let copies that are still in flight land before the CTA may exit.
+__device__ __forceinline__ void drain_delay() {
+  const unsigned long long t0 = global_ns();
+  while (global_ns() - t0 < kDrainNs) {}
 }
 
+// Tiled 2-D TMA load into this CTA's shared memory; completion bytes are signalled on
+// `bar` (a shared::cluster address).  With kCta == 2 the barrier may belong to the peer
+// CTA of the pair, which the cta_group::2 form permits.
+template <int kCta>
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
+  if (kCta == 1) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+  } else {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
+        "[%0], [%1, {%3, %4}], [%2];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
+        : "memory");
+  }
+}
+
+template <int kCta>
 __device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  if (kCta == 1)
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
+  else
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
 }
+template <int kCta>
 __device__ __forceinline__ void tmem_relinquish() {
-  asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  if (kCta == 1)
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  else
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
 }
+template <int kCta>
 __device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+  if (kCta == 1)
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
+  else
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate.
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate.  With kCta == 2 the
+// instruction runs on both SMs of the pair: each uses its own A rows and accumulator,
+// and B is the concatenation of the two CTAs' halves.
+template <int kCta>
 __device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
                                           uint32_t accumulate) {
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "setp.ne.b32 p, %4, 0;\n\t"
-      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-      : "memory");
+  if (kCta == 1) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  } else {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+  }
 }
-// Arrive on an mbarrier once every MMA issued so far by this thread has completed.
+// Arrive on an mbarrier once every MMA issued so far by this thread has completed.  With
+// kCta == 2 the arrival is delivered to the barrier at the same offset in both CTAs.
+template <int kCta>
 __device__ __forceinline__ void umma_commit(uint32_t bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  if (kCta == 1) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+  } else {
+    const uint16_t mask = 3;
+    asm volatile(
+        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+        ::"r"(bar), "h"(mask)
+        : "memory");
+  }
 }
 
 // 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i).
@@ -164,35 +250,40 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
   return dsc;
 }
 
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = n_cols.
-__device__ __forceinline__ uint32_t instr_desc(int n_cols) {
+// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = m_rows, N = n_cols.
+__device__ __forceinline__ uint32_t instr_desc(int m_rows, int n_cols) {
   return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n_cols >> 3) << 17) |
-         (static_cast<uint32_t>(kBlockM >> 4) << 24);
+         (static_cast<uint32_t>(m_rows >> 4) << 24);
 }
 
-struct UnitRange {
-  int row0;      // first token row of the unit
-  int g0, g1;    // granule range of the chunk
+// The static schedule, identical in every role: worker w walks units w, w + workers, ...;
+// each unit is `tiles_per_unit` tiles (possibly empty ones when the chunk is short).
+struct Tile {
+  int row0;    // first token row of this CTA in the unit
+  int chunk;
+  int v0;      // first vocabulary row of the tile
+  int rows;    // vocabulary rows in the tile (multiple of 16 * kCta); 0 = empty tile
 };
 
-__device__ __forceinline__ UnitRange unit_range(const TcParams& p, int unit) {
-  UnitRange u;
-  const int chunk = unit / p.row_units;
-  const int ru = unit - chunk * p.row_units;
-  u.row0 = ru * kBlockM;
-  u.g0 = static_cast<int>((static_cast<long long>(p.granules) * chunk) / p.chunks);
-  u.g1 = static_cast<int>((static_cast<long long>(p.granules) * (chunk + 1)) / p.chunks);
-  return u;
-}
-
-// Tile t of a chunk of G granules split as evenly as possible into T tiles.
-__device__ __forceinline__ void tile_range(int G, int T, int t, int* a, int* b) {
-  *a = (G * t) / T;
-  *b = (G * (t + 1)) / T;
+template <int kCta>
+__device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int cta_rank) {
+  Tile r;
+  r.chunk = unit / p.row_units;
+  const int ru = unit - r.chunk * p.row_units;
+  r.row0 = (ru * kCta + cta_rank) * kBlockM;
+  const int g0 = static_cast<int>((static_cast<long long>(p.granules) * r.chunk) / p.chunks);
+  const int g1 = static_cast<int>((static_cast<long long>(p.granules) * (r.chunk + 1)) / p.chunks);
+  const int G = g1 - g0;
+  const int ga = (G * t) / p.tiles_per_unit;
+  const int gb = (G * (t + 1)) / p.tiles_per_unit;
+  r.v0 = (g0 + ga) * (16 * kCta);
+  r.rows = (gb - ga) * (16 * kCta);
+  return r;
 }
 
 }  // namespace
 
+template <int kCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
                      const __grid_constant__ CUtensorMap map_w64,
@@ -200,154 +291,175 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
                      const TcParams p) {
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the shared-memory address.
+  // (The dynamic shared memory of both CTAs of a pair starts at the same offset, so the
+  // two CTAs compute identical offsets -- which the pair MMA and the peer signals rely on.)
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar_base = base + kStages * kStageBytes;
-  // barrier block: full[kStages], empty[kStages], acc_full[2], acc_empty[2], then tmem slot + abort flag
-  auto full_bar = [&](int s) { return bar_base + 8u * s; };
-  auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
-  auto acc_full_bar = [&](int b) { return bar_base + 8u * (2 * kStages + b); };
-  auto acc_empty_bar = [&](int b) { return bar_base + 8u * (2 * kStages + 2 + b); };
+  const int SA = p.a_stages, SB = p.b_stages;
+  const uint32_t a_stage_bytes = static_cast<uint32_t>(p.a_rows) * kRowBytes;
+  constexpr uint32_t b_stage_bytes = (kBlockN / kCta) * kRowBytes;
+  const uint32_t a_ring = base;
+  const uint32_t b_ring = base + SA * a_stage_bytes;
+  const uint32_t bar_base = b_ring + SB * b_stage_bytes;
+  auto a_full = [&](int s) { return bar_base + 8u * s; };
+  auto a_empty = [&](int s) { return bar_base + 8u * (kMaxAStages + s); };
+  auto b_full = [&](int s) { return bar_base + 8u * (2 * kMaxAStages + s); };
+  auto b_empty = [&](int s) { return bar_base + 8u * (2 * kMaxAStages + kMaxBStages + s); };
+  auto acc_full = [&](int b) { return bar_base + 8u * (2 * kMaxAStages + 2 * kMaxBStages + b); };
+  auto acc_empty = [&](int b) { return bar_base + 8u * (2 * kMaxAStages + 2 * kMaxBStages + 2 + b); };
+  constexpr int kNumBarriers = 2 * kMaxAStages + 2 * kMaxBStages + 4;
+  static_assert(kNumBarriers * 8 + 16 <= kBarrierBytes, "barrier block too small");
   unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + kStages * kStageBytes + 8 * (2 * kStages + 4));
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (bar_base - base) + 8 * kNumBarriers);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
+  const uint32_t cta_rank = (kCta == 2) ? cluster_ctarank() : 0u;
+  const bool leader = cta_rank == 0;
+  const int worker = blockIdx.x / kCta;
+  const int workers = gridDim.x / kCta;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kStages; ++s) {
-      mbar_init(full_bar(s), 1);
-      mbar_init(empty_bar(s), 1);
+    for (int s = 0; s < SA; ++s) {
+      mbar_init(a_full(s), 1);
+      mbar_init(a_empty(s), 1);
+    }
+    for (int s = 0; s < SB; ++s) {
+      mbar_init(b_full(s), 1);
+      mbar_init(b_empty(s), 1);
     }
     for (int b = 0; b < 2; ++b) {
-      mbar_init(acc_full_bar(b), 1);
-      mbar_init(acc_empty_bar(b), kEpiWarps);
+      mbar_init(acc_full(b), 1);
+      mbar_init(acc_empty(b), kEpiWarps * kCta);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
   if (warp == 1) {
-    tmem_alloc(smem_u32(tmem_slot), kTmemCols);
-    tmem_relinquish();
+    tmem_alloc<kCta>(smem_u32(tmem_slot), kTmemCols);
+    tmem_relinquish<kCta>();
   }
   tc_fence_before();
   __syncthreads();
+  if (kCta == 2) cluster_sync_all();   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
   const int k_slabs = (p.d + kBlockK - 1) / kBlockK;
   const int units = p.chunks * p.row_units;
+  const int T = p.tiles_per_unit;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ W producer
     if (lane == 0) {
       int stage = 0;
       uint32_t phase = 0;
-      int issued = 0;  // slabs issued in total
       bool ok = true;
-      for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x) {
-        const UnitRange u = unit_range(p, unit);
-        const int G = u.g1 - u.g0;
-        const int T = (G * 16 + kBlockN - 1) / kBlockN;
+      for (int unit = worker; unit < units && ok; unit += workers) {
         for (int t = 0; t < T && ok; ++t) {
-          int ga, gb;
-          tile_range(G, T, t, &ga, &gb);
-          const int v0 = (u.g0 + ga) * 16;
-          const int rows = (gb - ga) * 16;
+          const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+          if (tl.rows == 0) continue;
+          const int my_rows = tl.rows / kCta;                 // this CTA's share of the tile
+          const int my_v0 = tl.v0 + static_cast<int>(cta_rank) * my_rows;
           for (int ks = 0; ks < k_slabs; ++ks) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
-            const uint32_t sa = base + stage * kStageBytes;
-            const uint32_t sb = sa + kABytes;
-            mbar_expect_tx(full_bar(stage), kABytes + rows * (kBlockK * 2));
-            tma_load_2d(sa, &map_h, full_bar(stage), ks * kBlockK, u.row0);
+            if (!mbar_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t dst = b_ring + stage * b_stage_bytes;
+            const uint32_t bar = (kCta == 2) ? map_to_cta(b_full(stage), 0) : b_full(stage);
+            if (leader) mbar_expect_tx(b_full(stage), tl.rows * kRowBytes);   // both CTAs' bytes
             int r = 0;
-            for (; rows - r >= 64; r += 64)
-              tma_load_2d(sb + r * (kBlockK * 2), &map_w64, full_bar(stage), ks * kBlockK, v0 + r);
-            for (; rows - r >= 16; r += 16)
-              tma_load_2d(sb + r * (kBlockK * 2), &map_w16, full_bar(stage), ks * kBlockK, v0 + r);
-            ++issued;
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            for (; my_rows - r >= 64; r += 64)
+              tma_load_2d<kCta>(dst + r * kRowBytes, &map_w64, bar, ks * kBlockK, my_v0 + r);
+            for (; my_rows - r >= 16; r += 16)
+              tma_load_2d<kCta>(dst + r * kRowBytes, &map_w16, bar, ks * kBlockK, my_v0 + r);
+            if (++stage == SB) { stage = 0; phase ^= 1u; }
           }
         }
       }
-      if (!ok) {
-        // Drain: wait (bounded) until every slab already issued has landed, so that no
-        // copy is still writing shared memory when the CTA exits.
-        const int pending = issued < kStages ? issued : kStages;
-        int s = stage;
-        uint32_t ph = phase;
-        for (int i = 0; i < pending; ++i) {
-          if (--s < 0) { s = kStages - 1; ph ^= 1u; }
-          const unsigned long long t0 = global_ns();
-          while (!mbar_try_wait(full_bar(s), ph) && global_ns() - t0 < kWaitLimitNs) {}
+      if (!ok) drain_delay();
+    }
+  } else if (warp == 6) {
+    // ------------------------------------------------------------------ h producer
+    if (lane == 0) {
+      int stage = 0;
+      uint32_t phase = 0;
+      bool ok = true;
+      for (int unit = worker; unit < units && ok; unit += workers) {
+        for (int t = 0; t < T && ok; ++t) {
+          const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+          if (tl.rows == 0) continue;
+          for (int ks = 0; ks < k_slabs; ++ks) {
+            if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+            const uint32_t dst = a_ring + stage * a_stage_bytes;
+            const uint32_t bar = (kCta == 2) ? map_to_cta(a_full(stage), 0) : a_full(stage);
+            if (leader) mbar_expect_tx(a_full(stage), a_stage_bytes * kCta);
+            tma_load_2d<kCta>(dst, &map_h, bar, ks * kBlockK, tl.row0);
+            if (++stage == SA) { stage = 0; phase ^= 1u; }
+          }
         }
       }
+      if (!ok) drain_delay();
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      int stage = 0;
-      uint32_t phase = 0;
+    if (lane == 0 && leader) {
+      int sa = 0, sb = 0;
+      uint32_t pa = 0, pb = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
-      for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x) {
-        const UnitRange u = unit_range(p, unit);
-        const int G = u.g1 - u.g0;
-        const int T = (G * 16 + kBlockN - 1) / kBlockN;
+      for (int unit = worker; unit < units && ok; unit += workers) {
         for (int t = 0; t < T && ok; ++t) {
-          int ga, gb;
-          tile_range(G, T, t, &ga, &gb);
-          const uint32_t idesc = instr_desc((gb - ga) * 16);
-          if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          const Tile tl = tile_of<kCta>(p, unit, t, 0);
+          if (tl.rows == 0) continue;
+          const uint32_t idesc = instr_desc(kBlockM * kCta, tl.rows);
+          if (!mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * kBlockN;
           for (int ks = 0; ks < k_slabs; ++ks) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(a_full(sa), pa, abort_flag, p.status)) { ok = false; break; }
+            if (!mbar_wait(b_full(sb), pb, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            const uint32_t sa = base + stage * kStageBytes;
-            const uint64_t a_desc = smem_desc_sw128(sa);
-            const uint64_t b_desc = smem_desc_sw128(sa + kABytes);
+            const uint64_t a_desc = smem_desc_sw128(a_ring + sa * a_stage_bytes);
+            const uint64_t b_desc = smem_desc_sw128(b_ring + sb * b_stage_bytes);
 #pragma unroll
             for (int k = 0; k < kBlockK / kUmmaK; ++k) {
               // advancing 16 elements along K inside the swizzle span = +32 bytes = +2 in the address field
-              umma_bf16(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (ks | k) != 0 ? 1u : 0u);
+              umma_bf16<kCta>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (ks | k) != 0 ? 1u : 0u);
             }
-            umma_commit(empty_bar(stage));  // frees the slab once these MMAs have read it
-            if (++stage == kStages) { stage = 0; phase ^= 1u; }
+            umma_commit<kCta>(a_empty(sa));   // frees the slabs once these MMAs have read them
+            umma_commit<kCta>(b_empty(sb));
+            if (++sa == SA) { sa = 0; pa ^= 1u; }
+            if (++sb == SB) { sb = 0; pb ^= 1u; }
           }
           if (!ok) break;
-          umma_commit(acc_full_bar(acc));   // accumulator complete
+          umma_commit<kCta>(acc_full(acc));   // accumulator complete (in both CTAs of a pair)
           if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue
+    // ------------------------------------------------------------------ epilogue (warps 2-5)
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-    const int row_in_unit = quad * 32 + lane;
+    const int row_in_cta = quad * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int unit = blockIdx.x; unit < units && ok; unit += gridDim.x) {
-      const UnitRange u = unit_range(p, unit);
-      const int chunk = unit / p.row_units;
-      const int G = u.g1 - u.g0;
-      const int T_tiles = (G * 16 + kBlockN - 1) / kBlockN;
-      const bool warp_has_rows = (u.row0 + quad * 32) < p.n;   // warp-uniform
+    for (int unit = worker; unit < units && ok; unit += workers) {
+      const Tile first = tile_of<kCta>(p, unit, 0, cta_rank);
+      const bool warp_has_rows = (first.row0 + quad * 32) < p.n;   // warp-uniform
       // Running summary of this thread's row over the unit.  S = sum 2^y and T = sum 2^y * y
       // with y = (z - m) * log2(e) <= 0; both are accumulated per 32-column group first and
       // then added with a compensated (Kahan) sum, so that one dominant term -- a confident
       // row has S ~ 1 with thousands of terms ~1e-8 after it -- does not swallow the rest.
-      float m = -INFINITY, S = 0.f, cS = 0.f, T = 0.f, cT = 0.f;
+      float m = -INFINITY, S = 0.f, cS = 0.f, Tq = 0.f, cT = 0.f;
       int idx = kNoToken;
-      for (int t = 0; t < T_tiles && ok; ++t) {
-        int ga, gb;
-        tile_range(G, T_tiles, t, &ga, &gb);
-        const int v0 = (u.g0 + ga) * 16;
-        const int cols = min((gb - ga) * 16, p.V - v0);   // valid columns of this tile
-        if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+      for (int t = 0; t < T && ok; ++t) {
+        const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+        if (tl.rows == 0) continue;
+        const int v0 = tl.v0;
+        const int cols = min(tl.rows, p.V - v0);   // valid columns of this tile
+        if (!mbar_wait(acc_full(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
         tc_fence_after();
         if (warp_has_rows) {
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kBlockN;
@@ -369,16 +481,16 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
               if (m != -INFINITY) {
                 const float dl = (cm - m) * kLog2e;       // > 0
                 const float sc = ex2_approx(-dl);
-                T = sc * (T - dl * S);
+                Tq = sc * (Tq - dl * S);
                 cT *= sc;
                 S *= sc;
                 cS *= sc;
               }
               m = cm;
-              int first = 31;
+              int first_j = 31;
 #pragma unroll
-              for (int j = 30; j >= 0; --j) first = (z[j] == cm) ? j : first;
-              idx = v0 + c0 + first;
+              for (int j = 30; j >= 0; --j) first_j = (z[j] == cm) ? j : first_j;
+              idx = v0 + c0 + first_j;
             }
             const float neg_ml = -m * kLog2e;
             float ls0 = 0.f, ls1 = 0.f, lt0 = 0.f, lt1 = 0.f;
@@ -401,47 +513,92 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
             }
             {
               const float a = (lt0 + lt1) - cT;
-              const float b = T + a;
-              cT = (b - T) - a;
-              T = b;
+              const float b = Tq + a;
+              cT = (b - Tq) - a;
+              Tq = b;
             }
           }
         }
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        if (lane == 0) {
+          if (kCta == 1) mbar_arrive(acc_empty(acc));
+          else mbar_arrive_cluster(map_to_cta(acc_empty(acc), 0));   // the leader's barrier
+        }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      if (ok && u.row0 + row_in_unit < p.n) {
+      if (ok && first.row0 + row_in_cta < p.n) {
         Partial out;
         out.m = m;
         out.idx = idx;
         out.s = S;
-        out.t = T * kLn2;              // sum e^(z-m) (z-m), back in nats
-        p.partials[static_cast<size_t>(u.row0 + row_in_unit) * p.chunks + chunk] = out;
+        out.t = Tq * kLn2;             // sum e^(z-m) (z-m), back in nats
+        p.partials[static_cast<size_t>(first.row0 + row_in_cta) * p.chunks + first.chunk] = out;
       }
     }
   }
 
   tc_fence_before();
   __syncthreads();
+  if (kCta == 2) cluster_sync_all();   // neither CTA frees TMEM or exits while the peer still works
   if (warp == 1) {
     tc_fence_after();
-    tmem_dealloc(tmem_base, kTmemCols);
+    tmem_dealloc<kCta>(tmem_base, kTmemCols);
   }
 }
 
-int tc_smem_bytes() { return kSmemBytes; }
 int tc_threads() { return kThreads; }
 
+// Ring depths and shared-memory size for a given n.  The h ring is short (L2 latency),
+// the W ring takes everything that is left (HBM latency).
+void tc_configure(int n, TcConfig* c) {
+  const int cta = n > kBlockM ? 2 : 1;
+  int a_rows = kBlockM;
+  if (cta == 1) {
+    a_rows = ((n + 15) / 16) * 16;
+    if (a_rows < 16) a_rows = 16;
+    if (a_rows > kBlockM) a_rows = kBlockM;
+  }
+  const int a_stage = a_rows * kRowBytes;
+  const int b_stage = (kBlockN / cta) * kRowBytes;
+  int sa = a_rows <= 64 ? 3 : (cta == 2 ? 3 : 2);
+  const int budget = kSmemLimit - 1024 - kBarrierBytes;
+  int sb = (budget - sa * a_stage) / b_stage;
+  if (sb > kMaxBStages) sb = kMaxBStages;
+  c->cta = cta;
+  c->a_rows = a_rows;
+  c->a_stages = sa;
+  c->b_stages = sb;
+  c->smem_bytes = 1024 + sa * a_stage + sb * b_stage + kBarrierBytes;
+}
+
 cudaError_t tc_prepare() {
-  return cudaFuncSetAttribute(tc_projection_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
+  cudaError_t e = cudaFuncSetAttribute(tc_projection_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kSmemLimit);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(tc_projection_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  return e;
 }
 
 cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w64, const CUtensorMap& map_w16,
-                                 const TcParams& p, int grid, cudaStream_t stream) {
-  tc_projection_kernel<<<grid, kThreads, kSmemBytes, stream>>>(map_h, map_w64, map_w16, p);
-  return cudaGetLastError();
+                                 const TcParams& p, const TcConfig& c, int workers, cudaStream_t stream) {
+  if (c.cta == 1) {
+    tc_projection_kernel<1><<<workers, kThreads, c.smem_bytes, stream>>>(map_h, map_w64, map_w16, p);
+    return cudaGetLastError();
+  }
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(workers * 2), 1, 1);
+  cfg.blockDim = dim3(kThreads, 1, 1);
+  cfg.dynamicSmemBytes = static_cast<size_t>(c.smem_bytes);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = 2;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2>, map_h, map_w64, map_w16, p);
 }
 
 }  // namespace tlr

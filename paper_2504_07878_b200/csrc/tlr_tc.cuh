@@ -7,23 +7,37 @@
 
 namespace tlr {
 
+// Kernel shape for a given n (see tc_configure).
+struct TcConfig {
+  int cta;          // 1: one CTA per worker (n <= 128); 2: a pair of CTAs per worker
+  int a_rows;       // rows of an h slab held in shared memory (16..128)
+  int a_stages;     // depth of the h ring
+  int b_stages;     // depth of the W ring
+  int smem_bytes;   // dynamic shared memory per CTA
+};
+
+// Work decomposition for a given (n, V) on `workers` workers (see tc_plan).
+struct TcPlan {
+  int row_units;       // ceil(n / (128 * cta))
+  int chunks;          // vocabulary chunks == partials per row
+  int granule_rows;    // 16 * cta
+  int granules;        // ceil(V / granule_rows)
+  int tiles_per_unit;  // every unit is walked in this many tiles (<= 256 rows each)
+};
+
 struct TcParams {
   int n, d, V;
-  int row_units;    // ceil(n / 128)
-  int chunks;       // vocabulary chunks == partials per row
-  int granules;     // ceil(V / 16): the vocabulary in 16-row granules
+  int row_units, chunks, granules, tiles_per_unit;
+  int a_rows, a_stages, b_stages;
   Partial* partials;  // [n][chunks]
   uint32_t* status;
 };
 
-int tc_smem_bytes();
 int tc_threads();
-cudaError_t tc_prepare();   // opt in to the kernel's dynamic shared memory size (once per device)
+void tc_configure(int n, TcConfig* c);
+void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan);
+cudaError_t tc_prepare();   // opt in to the kernels' dynamic shared memory size (once per device)
 cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w64, const CUtensorMap& map_w16,
-                                 const TcParams& p, int grid, cudaStream_t stream);
-
-// Chooses the number of vocabulary chunks for n rows on `workers` CTAs: the count that
-// minimises (waves of units) x (rows per chunk + a fixed per-unit cost), capped at max_chunks.
-int tc_choose_chunks(int n, int V, int workers, int max_chunks);
+                                 const TcParams& p, const TcConfig& c, int workers, cudaStream_t stream);
 
 }  // namespace tlr
