@@ -20,6 +20,11 @@ finish_kernel(const FinishLaunch a) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFinishWarps + warp;
+  // Programmatic dependent launch: let the next kernel in the stream be scheduled now (it
+  // waits for this grid to complete before touching memory), then wait for the projection
+  // kernel's partials.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 
   if (row < a.n) {
     const Partial* p = a.partials + (size_t)row * a.chunks;
@@ -94,8 +99,17 @@ finish_kernel(const FinishLaunch a) {
 
 cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream) {
   const int blocks = a.n > 0 ? (a.n + kFinishWarps - 1) / kFinishWarps : 1;
-  finish_kernel<<<blocks, kFinishThreads, 0, stream>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(kFinishThreads, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, finish_kernel, a);
 }
 
 }  // namespace tlr

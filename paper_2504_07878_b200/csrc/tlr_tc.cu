@@ -38,6 +38,9 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <cstdio>
+#include <cstdlib>
+
 #include "tlr_common.cuh"
 #include "tlr_tc.cuh"
 
@@ -53,8 +56,9 @@ constexpr int kRowBytes = kBlockK * 2;       // 128
 constexpr int kTmemCols = 512;
 constexpr int kEpiWarps = 4;
 constexpr int kThreads = 32 * 7;
-constexpr int kMaxAStages = 4;
+constexpr int kMaxAStages = 8;
 constexpr int kMaxBStages = 12;
+constexpr int kRelease = 16;                 // >= every ring depth (see the barrier notes in the kernel)
 constexpr int kBarrierBytes = 512;
 constexpr int kSmemLimit = 232448;           // 227 KiB opt-in maximum per CTA
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
@@ -104,6 +108,19 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
   asm volatile(
       "{\n\t.reg .pred p;\n\t"
       "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(bar), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+
+// Non-blocking poll of the same condition.
+__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
+  uint32_t ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
       "selp.u32 %0, 1, 0, p;\n\t}"
       : "=r"(ok)
       : "r"(bar), "r"(parity)
@@ -300,13 +317,16 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   const uint32_t a_ring = base;
   const uint32_t b_ring = base + SA * a_stage_bytes;
   const uint32_t bar_base = b_ring + SB * b_stage_bytes;
+  // Barriers: a_full / b_full per ring stage (data landed); released[j] completes when the
+  // MMAs of slab number j (mod kRelease) have finished reading shared memory -- one commit
+  // per slab serves both rings: the producer of slab i waits for slab i - depth;
+  // acc_full / acc_empty per accumulator.
   auto a_full = [&](int s) { return bar_base + 8u * s; };
-  auto a_empty = [&](int s) { return bar_base + 8u * (kMaxAStages + s); };
-  auto b_full = [&](int s) { return bar_base + 8u * (2 * kMaxAStages + s); };
-  auto b_empty = [&](int s) { return bar_base + 8u * (2 * kMaxAStages + kMaxBStages + s); };
-  auto acc_full = [&](int b) { return bar_base + 8u * (2 * kMaxAStages + 2 * kMaxBStages + b); };
-  auto acc_empty = [&](int b) { return bar_base + 8u * (2 * kMaxAStages + 2 * kMaxBStages + 2 + b); };
-  constexpr int kNumBarriers = 2 * kMaxAStages + 2 * kMaxBStages + 4;
+  auto b_full = [&](int s) { return bar_base + 8u * (kMaxAStages + s); };
+  auto released = [&](int j) { return bar_base + 8u * (kMaxAStages + kMaxBStages + j); };
+  auto acc_full = [&](int b) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + b); };
+  auto acc_empty = [&](int b) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + 2 + b); };
+  constexpr int kNumBarriers = kMaxAStages + kMaxBStages + kRelease + 4;
   static_assert(kNumBarriers * 8 + 16 <= kBarrierBytes, "barrier block too small");
   unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (bar_base - base) + 8 * kNumBarriers);
@@ -320,14 +340,9 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   const int workers = gridDim.x / kCta;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < SA; ++s) {
-      mbar_init(a_full(s), 1);
-      mbar_init(a_empty(s), 1);
-    }
-    for (int s = 0; s < SB; ++s) {
-      mbar_init(b_full(s), 1);
-      mbar_init(b_empty(s), 1);
-    }
+    for (int s = 0; s < SA; ++s) mbar_init(a_full(s), 1);
+    for (int s = 0; s < SB; ++s) mbar_init(b_full(s), 1);
+    for (int j = 0; j < kRelease; ++j) mbar_init(released(j), 1);
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full(b), 1);
       mbar_init(acc_empty(b), kEpiWarps * kCta);
@@ -345,6 +360,12 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   if (kCta == 2) cluster_sync_all();   // the peer's barriers exist before anything signals them
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Programmatic dependent launch: everything above overlapped the tail of the previous
+  // kernel in the stream; from here on its results (h, and the workspace the previous
+  // merge kernel was still reading) are needed, so wait for it, then let the merge kernel
+  // that follows this one be scheduled early.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int k_slabs = (p.d + kBlockK - 1) / kBlockK;
   const int units = p.chunks * p.row_units;
@@ -354,7 +375,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     // ------------------------------------------------------------------ W producer
     if (lane == 0) {
       int stage = 0;
-      uint32_t phase = 0;
+      int slab = 0;     // running slab number, the same in every role
       bool ok = true;
       for (int unit = worker; unit < units && ok; unit += workers) {
         for (int t = 0; t < T && ok; ++t) {
@@ -362,8 +383,11 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           if (tl.rows == 0) continue;
           const int my_rows = tl.rows / kCta;                 // this CTA's share of the tile
           const int my_v0 = tl.v0 + static_cast<int>(cta_rank) * my_rows;
-          for (int ks = 0; ks < k_slabs; ++ks) {
-            if (!mbar_wait(b_empty(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
+            if (slab >= SB) {     // the stage is free once slab - SB has been consumed
+              const int j = slab - SB;
+              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status)) { ok = false; break; }
+            }
             const uint32_t dst = b_ring + stage * b_stage_bytes;
             const uint32_t bar = (kCta == 2) ? map_to_cta(b_full(stage), 0) : b_full(stage);
             if (leader) mbar_expect_tx(b_full(stage), tl.rows * kRowBytes);   // both CTAs' bytes
@@ -372,7 +396,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
               tma_load_2d<kCta>(dst + r * kRowBytes, &map_w64, bar, ks * kBlockK, my_v0 + r);
             for (; my_rows - r >= 16; r += 16)
               tma_load_2d<kCta>(dst + r * kRowBytes, &map_w16, bar, ks * kBlockK, my_v0 + r);
-            if (++stage == SB) { stage = 0; phase ^= 1u; }
+            if (++stage == SB) stage = 0;
           }
         }
       }
@@ -382,19 +406,22 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     // ------------------------------------------------------------------ h producer
     if (lane == 0) {
       int stage = 0;
-      uint32_t phase = 0;
+      int slab = 0;
       bool ok = true;
       for (int unit = worker; unit < units && ok; unit += workers) {
         for (int t = 0; t < T && ok; ++t) {
           const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
           if (tl.rows == 0) continue;
-          for (int ks = 0; ks < k_slabs; ++ks) {
-            if (!mbar_wait(a_empty(stage), phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
+            if (slab >= SA) {
+              const int j = slab - SA;
+              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status)) { ok = false; break; }
+            }
             const uint32_t dst = a_ring + stage * a_stage_bytes;
             const uint32_t bar = (kCta == 2) ? map_to_cta(a_full(stage), 0) : a_full(stage);
             if (leader) mbar_expect_tx(a_full(stage), a_stage_bytes * kCta);
             tma_load_2d<kCta>(dst, &map_h, bar, ks * kBlockK, tl.row0);
-            if (++stage == SA) { stage = 0; phase ^= 1u; }
+            if (++stage == SA) stage = 0;
           }
         }
       }
@@ -405,9 +432,20 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     if (lane == 0 && leader) {
       int sa = 0, sb = 0;
       uint32_t pa = 0, pb = 0;
+      int slab = 0;
       int acc = 0;
       uint32_t acc_phase = 0;
       bool ok = true;
+      // Descriptor words: the low word carries the start address (in 16-byte units) and the
+      // leading offset; the high word is constant.
+      const uint64_t desc_hi = smem_desc_sw128(0) & 0xffffffff00000000ull;
+      const uint32_t desc_lo_fixed = static_cast<uint32_t>(smem_desc_sw128(0) & 0xffffffffull);
+      const uint32_t a_lo0 = desc_lo_fixed | ((a_ring & 0x3ffffu) >> 4);
+      const uint32_t b_lo0 = desc_lo_fixed | ((b_ring & 0x3ffffu) >> 4);
+      const uint32_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;
+      // The barrier state of the next slab is polled before the current slab's MMAs are
+      // issued, so the poll's latency overlaps the issue instead of adding to it.
+      bool ra = mbar_test_wait(a_full(0), 0), rb = mbar_test_wait(b_full(0), 0);
       for (int unit = worker; unit < units && ok; unit += workers) {
         for (int t = 0; t < T && ok; ++t) {
           const Tile tl = tile_of<kCta>(p, unit, t, 0);
@@ -416,21 +454,23 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           if (!mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * kBlockN;
-          for (int ks = 0; ks < k_slabs; ++ks) {
-            if (!mbar_wait(a_full(sa), pa, abort_flag, p.status)) { ok = false; break; }
-            if (!mbar_wait(b_full(sb), pb, abort_flag, p.status)) { ok = false; break; }
+          for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
+            if (!ra && !mbar_wait(a_full(sa), pa, abort_flag, p.status)) { ok = false; break; }
+            if (!rb && !mbar_wait(b_full(sb), pb, abort_flag, p.status)) { ok = false; break; }
             tc_fence_after();
-            const uint64_t a_desc = smem_desc_sw128(a_ring + sa * a_stage_bytes);
-            const uint64_t b_desc = smem_desc_sw128(b_ring + sb * b_stage_bytes);
+            const uint32_t a_lo = a_lo0 + sa * a_step;
+            const uint32_t b_lo = b_lo0 + sb * b_step;
+            if (++sa == SA) { sa = 0; pa ^= 1u; }
+            if (++sb == SB) { sb = 0; pb ^= 1u; }
+            ra = mbar_test_wait(a_full(sa), pa);
+            rb = mbar_test_wait(b_full(sb), pb);
 #pragma unroll
             for (int k = 0; k < kBlockK / kUmmaK; ++k) {
               // advancing 16 elements along K inside the swizzle span = +32 bytes = +2 in the address field
-              umma_bf16<kCta>(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (ks | k) != 0 ? 1u : 0u);
+              umma_bf16<kCta>(d_tmem, desc_hi | (a_lo + 2u * k), desc_hi | (b_lo + 2u * k), idesc,
+                              (ks | k) != 0 ? 1u : 0u);
             }
-            umma_commit<kCta>(a_empty(sa));   // frees the slabs once these MMAs have read them
-            umma_commit<kCta>(b_empty(sb));
-            if (++sa == SA) { sa = 0; pa ^= 1u; }
-            if (++sb == SB) { sb = 0; pb ^= 1u; }
+            umma_commit<kCta>(released(slab & (kRelease - 1)));   // both slabs are free once these MMAs are done
           }
           if (!ok) break;
           umma_commit<kCta>(acc_full(acc));   // accumulator complete (in both CTAs of a pair)
@@ -561,10 +601,21 @@ void tc_configure(int n, TcConfig* c) {
   }
   const int a_stage = a_rows * kRowBytes;
   const int b_stage = (kBlockN / cta) * kRowBytes;
-  int sa = a_rows <= 64 ? 3 : (cta == 2 ? 3 : 2);
+  // h slabs come from L2 (about a microsecond away under load) and one is consumed per W
+  // slab, so the h ring needs about half the depth of the W ring to keep up.
+  int sa = cta == 2 ? 5 : (a_rows <= 32 ? 6 : 4);
   const int budget = kSmemLimit - 1024 - kBarrierBytes;
   int sb = (budget - sa * a_stage) / b_stage;
   if (sb > kMaxBStages) sb = kMaxBStages;
+  // Tuning override: TLR_TC_RINGS="<h stages>,<W stages>" (ignored if it does not fit).
+  if (const char* env = getenv("TLR_TC_RINGS")) {
+    int ea = 0, eb = 0;
+    if (sscanf(env, "%d,%d", &ea, &eb) == 2 && ea >= 1 && ea <= kMaxAStages && eb >= 1 && eb <= kMaxBStages &&
+        ea * a_stage + eb * b_stage <= budget) {
+      sa = ea;
+      sb = eb;
+    }
+  }
   c->cta = cta;
   c->a_rows = a_rows;
   c->a_stages = sa;
@@ -582,22 +633,24 @@ cudaError_t tc_prepare() {
 
 cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w64, const CUtensorMap& map_w16,
                                  const TcParams& p, const TcConfig& c, int workers, cudaStream_t stream) {
-  if (c.cta == 1) {
-    tc_projection_kernel<1><<<workers, kThreads, c.smem_bytes, stream>>>(map_h, map_w64, map_w16, p);
-    return cudaGetLastError();
-  }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(workers * 2), 1, 1);
+  cfg.gridDim = dim3(static_cast<unsigned>(workers * c.cta), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
   cfg.dynamicSmemBytes = static_cast<size_t>(c.smem_bytes);
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
-  attr[0].id = cudaLaunchAttributeClusterDimension;
-  attr[0].val.clusterDim.x = 2;
-  attr[0].val.clusterDim.y = 1;
-  attr[0].val.clusterDim.z = 1;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = 2;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  if (c.cta == 1) {
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1>, map_h, map_w64, map_w16, p);
+  }
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2>, map_h, map_w64, map_w16, p);
 }
 
