@@ -1,62 +1,252 @@
 // Merge of the per-chunk partial results, the scores, the route decision and the
 // ordered stream compaction of routed rows -- one launch.
 //
-// Phase 1 (all blocks): one warp per row folds that row's `chunks` partials with the
-//   associative merge rule (lanes stride the partials, then a shuffle butterfly),
-//   and lane 0 writes token, conf = 1/s, entropy = ln s - t/s and the route flag
-//   conf < tau (Sec. 3.1 of the paper: routed when the score falls below the threshold).
-// Phase 2 (the block that finishes last, found with a fence + ticket counter, no
-//   spinning): ballot / popcount / prefix-sum compaction of the flags into the
-//   ascending index list, and the count.
+// Per row (one warp): lanes stride the row's partials; a shuffle butterfly finds the
+// global maximum and its lowest index, each lane rescales its own partials to that
+// maximum once, and a second butterfly adds the sums.  Lane 0 writes token,
+// conf = 1/s, entropy = ln s - t/s and the route flag conf < tau (Sec. 3.1 of the
+// paper: routed when the score falls below the threshold).
+//
+// Compaction (ballot / popcount / prefix sum, ascending order):
+//   n <= 1024  a thread-block cluster of up to 8 blocks folds the rows (a group of L lanes
+//              per row, all rows at once); after a cluster barrier block 0 compacts the
+//              flags in one pass.  No ticket, no second launch, about two L2 round trips.
+//   larger n   many blocks of 8 warps; the block that finishes last (fence + ticket
+//              counter, no spinning) compacts the flags of all rows.
 #include "tlr_common.cuh"
 
 namespace tlr {
 
 constexpr int kFinishWarps = 8;
 constexpr int kFinishThreads = kFinishWarps * 32;
+constexpr int kSmallThreads = 1024;
+constexpr int kSmallRows = 1024;
+constexpr int kPerLane = 6;            // ceil(192 / 32): the most partials a lane can own
+
+// Folds one row's partials.  Every lane returns the same result.
+__device__ __forceinline__ Partial fold_row(const Partial* __restrict__ p, int chunks, int lane) {
+  Partial q[kPerLane];
+  float m = -INFINITY;
+  int idx = kNoToken;
+#pragma unroll
+  for (int k = 0; k < kPerLane; ++k) {
+    const int j = lane + 32 * k;
+    if (j < chunks) {
+      const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+      q[k].m = raw.x;
+      q[k].idx = __float_as_int(raw.y);
+      q[k].s = raw.z;
+      q[k].t = raw.w;
+    } else {
+      q[k] = empty_partial();
+    }
+    if (q[k].m > m || (q[k].m == m && q[k].idx < idx)) {
+      m = q[k].m;
+      idx = q[k].idx;
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    const float om = __shfl_xor_sync(0xffffffffu, m, off);
+    const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+    if (om > m || (om == m && oi < idx)) {
+      m = om;
+      idx = oi;
+    }
+  }
+  float s = 0.f, t = 0.f;
+#pragma unroll
+  for (int k = 0; k < kPerLane; ++k) {
+    if (!(q[k].s == 0.f)) {           // an empty range contributes nothing; a NaN sum goes through
+      const float dm = q[k].m - m;    // <= 0
+      const float e = exp2f(dm * kLog2e);
+      s += q[k].s * e;
+      t += e * (q[k].t + dm * q[k].s);
+    }
+  }
+#pragma unroll
+  for (int off = 16; off > 0; off >>= 1) {
+    s += __shfl_xor_sync(0xffffffffu, s, off);
+    t += __shfl_xor_sync(0xffffffffu, t, off);
+  }
+  Partial r;
+  r.m = m;
+  r.idx = idx;
+  r.s = s;
+  r.t = t;
+  return r;
+}
+
+// Scores and decision of one row from its folded summary; returns the route flag.
+__device__ __forceinline__ int score_row(const Partial& acc, const FinishLaunch& a, int row) {
+  float conf = 1.0f / acc.s;
+  float ent = logf(acc.s) - acc.t / acc.s;
+  const bool finite = (conf == conf) && (ent == ent) && acc.s > 0.f && acc.s < INFINITY;
+  if (finite) {
+    conf = fminf(conf, 1.0f);
+    ent = fmaxf(ent, 0.0f);
+  } else {
+    conf = __int_as_float(0x7fc00000);   // NaN: fails "conf >= tau", so the row is routed
+    ent = conf;
+    atomicOr(a.status, TLR_DEV_NONFINITE);
+  }
+  // "not (conf >= tau)": equals conf < tau for numbers, and routes a NaN row.
+  const int flag = (conf >= a.tau) ? 0 : 1;
+  a.token[row] = acc.idx;
+  a.conf[row] = conf;
+  a.entropy[row] = ent;
+  a.route_mask[row] = static_cast<uint8_t>(flag);
+  return flag;
+}
+
+// Programmatic dependent launch: let the next kernel in the stream be scheduled now (it
+// waits for this grid to complete before touching memory), then wait for the projection
+// kernel's partials.
+__device__ __forceinline__ void pdl_enter() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+}
+
+// Cluster of gridDim.x blocks, n <= 1024.  A group of L lanes (L a power of two) folds one
+// row in two passes over its partials: maximum and index first, then the sums rescaled to
+// that maximum.  L is chosen on the host so that every row has its group: n * L <=
+// gridDim.x * 1024.
+__global__ void __launch_bounds__(kSmallThreads)
+finish_small_kernel(const FinishLaunch a, const int L) {
+  __shared__ int warp_count[kSmallThreads / 32];
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const int group = (blockIdx.x * kSmallThreads + threadIdx.x) / L;
+  const int gl = threadIdx.x & (L - 1);
+  pdl_enter();
+  __shared__ unsigned char flags[kSmallRows];
+  const bool single_block = gridDim.x == 1;
+  {
+    const int row = group;
+    const bool valid = row < a.n;
+    const Partial* p = a.partials + static_cast<size_t>(valid ? row : 0) * a.chunks;
+    float m = -INFINITY;
+    int idx = kNoToken;
+    float s = 0.f, t = 0.f;
+    if ((a.chunks + L - 1) / L <= kPerLane) {
+      // few partials per lane: one pass, the partials stay in registers
+      Partial q[kPerLane];
+#pragma unroll
+      for (int k = 0; k < kPerLane; ++k) {
+        const int j = gl + L * k;
+        if (valid && j < a.chunks) {
+          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+          q[k].m = raw.x;
+          q[k].idx = __float_as_int(raw.y);
+          q[k].s = raw.z;
+          q[k].t = raw.w;
+        } else {
+          q[k] = empty_partial();
+        }
+        if (q[k].m > m || (q[k].m == m && q[k].idx < idx)) {
+          m = q[k].m;
+          idx = q[k].idx;
+        }
+      }
+      for (int off = L >> 1; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+        if (om > m || (om == m && oi < idx)) {
+          m = om;
+          idx = oi;
+        }
+      }
+#pragma unroll
+      for (int k = 0; k < kPerLane; ++k) {
+        if (!(q[k].s == 0.f)) {         // an empty range contributes nothing; a NaN sum goes through
+          const float dm = q[k].m - m;  // <= 0
+          const float e = exp2f(dm * kLog2e);
+          s += q[k].s * e;
+          t += e * (q[k].t + dm * q[k].s);
+        }
+      }
+    } else {
+      // many partials per lane: maximum and index first, then the rescaled sums
+      if (valid) {
+        for (int j = gl; j < a.chunks; j += L) {
+          const float2 mi = __ldcg(reinterpret_cast<const float2*>(p + j));
+          const int qi = __float_as_int(mi.y);
+          if (mi.x > m || (mi.x == m && qi < idx)) {
+            m = mi.x;
+            idx = qi;
+          }
+        }
+      }
+      for (int off = L >> 1; off > 0; off >>= 1) {
+        const float om = __shfl_xor_sync(0xffffffffu, m, off);
+        const int oi = __shfl_xor_sync(0xffffffffu, idx, off);
+        if (om > m || (om == m && oi < idx)) {
+          m = om;
+          idx = oi;
+        }
+      }
+      if (valid) {
+        for (int j = gl; j < a.chunks; j += L) {
+          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+          if (!(raw.z == 0.f)) {
+            const float dm = raw.x - m;
+            const float e = exp2f(dm * kLog2e);
+            s += raw.z * e;
+            t += e * (raw.w + dm * raw.z);
+          }
+        }
+      }
+    }
+    for (int off = L >> 1; off > 0; off >>= 1) {
+      s += __shfl_xor_sync(0xffffffffu, s, off);
+      t += __shfl_xor_sync(0xffffffffu, t, off);
+    }
+    if (valid && gl == 0) {
+      Partial acc;
+      acc.m = m;
+      acc.idx = idx;
+      acc.s = s;
+      acc.t = t;
+      const int f = score_row(acc, a, row);
+      if (single_block) flags[row] = static_cast<unsigned char>(f);
+    }
+  }
+  if (single_block) {
+    __syncthreads();                    // the flags are in this block's shared memory
+  } else {
+    // Every block's flags are in route_mask; the cluster barrier (release / acquire) makes
+    // them visible to block 0, which compacts them.
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+  }
+  if (blockIdx.x != 0) return;
+  const int i = threadIdx.x;
+  int flag = 0;
+  if (i < a.n) flag = single_block ? static_cast<int>(flags[i]) : static_cast<int>(__ldcg(a.route_mask + i));
+  const unsigned int bal = __ballot_sync(0xffffffffu, flag != 0);
+  if (lane == 0) warp_count[warp] = __popc(bal);
+  __syncthreads();
+  int before = 0, total = 0;
+#pragma unroll
+  for (int w = 0; w < kSmallThreads / 32; ++w) {
+    const int c = warp_count[w];
+    before += (w < warp) ? c : 0;
+    total += c;
+  }
+  if (flag) a.routed_idx[before + __popc(bal & ((1u << lane) - 1u))] = i;
+  if (threadIdx.x == 0) *a.routed_count = total;
+}
 
 __global__ void __launch_bounds__(kFinishThreads)
 finish_kernel(const FinishLaunch a) {
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFinishWarps + warp;
-  // Programmatic dependent launch: let the next kernel in the stream be scheduled now (it
-  // waits for this grid to complete before touching memory), then wait for the projection
-  // kernel's partials.
-  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  pdl_enter();
 
   if (row < a.n) {
-    const Partial* p = a.partials + (size_t)row * a.chunks;
-    Partial acc = empty_partial();
-    for (int j = lane; j < a.chunks; j += 32) {
-      const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
-      Partial q;
-      q.m = raw.x;
-      q.idx = __float_as_int(raw.y);
-      q.s = raw.z;
-      q.t = raw.w;
-      acc = merge(acc, q);
-    }
-    acc = warp_merge(acc);
-    if (lane == 0) {
-      float conf = 1.0f / acc.s;
-      float ent = logf(acc.s) - acc.t / acc.s;
-      const bool finite = (conf == conf) && (ent == ent) && acc.s > 0.f && acc.s < INFINITY;
-      if (finite) {
-        conf = fminf(conf, 1.0f);
-        ent = fmaxf(ent, 0.0f);
-      } else {
-        conf = __int_as_float(0x7fc00000);   // NaN: fails "conf >= tau", so the row is routed
-        ent = conf;
-        atomicOr(a.status, TLR_DEV_NONFINITE);
-      }
-      a.token[row] = acc.idx;
-      a.conf[row] = conf;
-      a.entropy[row] = ent;
-      // "not (conf >= tau)": equals conf < tau for numbers, and routes a NaN row.
-      a.route_mask[row] = (conf >= a.tau) ? 0 : 1;
-    }
+    const Partial acc = fold_row(a.partials + static_cast<size_t>(row) * a.chunks, a.chunks, lane);
+    if (lane == 0) score_row(acc, a, row);
   }
 
   // ---- which block is last?
@@ -98,17 +288,32 @@ finish_kernel(const FinishLaunch a) {
 }
 
 cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream) {
-  const int blocks = a.n > 0 ? (a.n + kFinishWarps - 1) / kFinishWarps : 1;
+  if (a.chunks > 32 * kPerLane) return cudaErrorInvalidValue;
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-  cfg.blockDim = dim3(kFinishThreads, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = stream;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
+  if (a.n <= kSmallRows) {
+    int blocks = 1;
+    while (blocks < 8 && blocks * 32 < a.n) blocks <<= 1;       // 32 rows per block until 8 blocks
+    int L = 32;
+    while (L > 1 && a.n * L > blocks * kSmallThreads) L >>= 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;
+    attr[1].val.clusterDim.x = static_cast<unsigned>(blocks);
+    attr[1].val.clusterDim.y = 1;
+    attr[1].val.clusterDim.z = 1;
+    cfg.numAttrs = 2;
+    cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+    cfg.blockDim = dim3(kSmallThreads, 1, 1);
+    return cudaLaunchKernelEx(&cfg, finish_small_kernel, a, L);
+  }
+  const int blocks = (a.n + kFinishWarps - 1) / kFinishWarps;
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(kFinishThreads, 1, 1);
   return cudaLaunchKernelEx(&cfg, finish_kernel, a);
 }
 
