@@ -31,6 +31,27 @@ UNIT = "tokens/s"
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reported against the HBM roofline
 
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the projection kernel, from the ncu
+# captures summarised under profiles/.  Only valid for the kernel source they were taken on: the
+# hash of that source is recorded here and traffic is reported as null when the source differs.
+NCU_TRAFFIC = {
+    "kernel_source": "paper_2504_07878_b200/csrc/tlr_tc.cu",
+    "sha256": "2f5ad762fe08c2e7344f78b141a4651eae56680604f18d26bb3464642656c7bb",
+    "bytes_per_launch": {"decode256": 276.68e6, "decode16": 276.32e6, "sweep512": 533.06e6},
+}
+
+
+def ncu_traffic(workload):
+    import hashlib
+    path = os.path.join(ROOT, NCU_TRAFFIC["kernel_source"])
+    try:
+        with open(path, "rb") as f:
+            if hashlib.sha256(f.read()).hexdigest() != NCU_TRAFFIC["sha256"]:
+                return None
+    except OSError:
+        return None
+    return NCU_TRAFFIC["bytes_per_launch"].get(workload)
+
 
 def measured_peaks():
     path = os.path.join(ROOT, "MEASURED_PEAKS.json")
@@ -229,7 +250,8 @@ def run_ours(args):
         achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained" if ms_total > 1000 else "bf16_tflops", peaks["bf16_tflops"]))
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s"}
-    roof.update({"frac": achieved / peak, "traffic": None, "peak_source": "of " + peak_kind,
+    roof.update({"frac": achieved / peak, "traffic": ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V),
+                 "peak_source": "of " + peak_kind,
                  "kernel": "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel",
                  "kernel_ms": kernel_ms, "kernel_launches_timed": launches,
                  "tensor_frac_same_launch": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
