@@ -109,6 +109,21 @@ class ClockSampler:
                 "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
 
 
+def max_over_ranks(x, world, device):
+    """The slowest rank's time decides the job's throughput (works on nccl and gloo groups)."""
+    if world <= 1:
+        return float(x)
+    import torch.distributed as dist
+    t = torch.tensor([float(x)], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_throughput(world, rows_per_rank, seconds_per_step):
+    """Weak scaling: every rank routes its own rows_per_rank rows per step."""
+    return world * rows_per_rank / seconds_per_step
+
+
 def physical_gpu_index(local_rank):
     vis = os.environ.get("CUDA_VISIBLE_DEVICES")
     if vis:
@@ -180,12 +195,7 @@ def run_ours(args):
         time.sleep(0.002)
     sampler.sample()
     barrier()
-    ms_total = e0.elapsed_time(e1)
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([ms_total], device="cuda")
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_total = float(t.item())
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
     status = max(P.tlr_last_device_status(r.ctx) for r in routers)
     if status & P.TLR_DEV_WAIT_TIMEOUT:
         raise SystemExit("device status flags raised during the timed region: %d" % status)
@@ -226,12 +236,7 @@ def run_ours(args):
     for i in range(esteps):
         host_step(i)
     torch.cuda.synchronize()
-    e2e_s = time.perf_counter() - t0
-    if world > 1:
-        import torch.distributed as dist
-        t = torch.tensor([e2e_s], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        e2e_s = float(t.item())
+    e2e_s = max_over_ranks(time.perf_counter() - t0, world, "cuda")
     e2e_routed = int(o_cnt.item())
     h2d = n * d * 2
     d2h = n * (4 + 4 + 4 + 1) + 4 + 4 + 4 * e2e_routed      # + status word + routed_idx[:count]
@@ -240,7 +245,7 @@ def run_ours(args):
         return
     peaks, peak_kind = measured_peaks()
     ms_per_step = ms_total / args.steps
-    value = world * n / (ms_per_step * 1e-3)
+    value = job_throughput(world, n, ms_per_step * 1e-3)
     hbm_bound = n <= RIDGE_ROWS_HBM
     if hbm_bound:
         achieved = algorithmic_bytes(n, d, V) / (kernel_ms * 1e-3) / 1e9
@@ -270,7 +275,7 @@ def run_ours(args):
                          % (2 * V * d / 1e6),
                    "path": int(plan.path), "grid": int(plan.grid), "block": int(plan.block),
                    "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed},
-        "e2e": {"value": world * n * esteps / e2e_s, "unit": UNIT, "h2d_bytes_per_step": h2d,
+        "e2e": {"value": job_throughput(world, n, e2e_s / esteps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)"},
         "gpu_launches": int(plan.launches) * args.steps,
         "clocks": sampler.summary(),
