@@ -159,6 +159,8 @@ def run_ours(args):
     wl = S.WORKLOADS[args.workload]
     n, d, V = wl.n, wl.d, wl.V
     tau = 0.5 if wl.tau is None else wl.tau
+    if args.tau is not None:
+        tau = args.tau
     W_host = S.make_W(d, V, seed=0)
     hid = S.make_h(n, d, seed=rank, W=W_host, planted_fraction=wl.planted_fraction)
     # two device copies of W, alternated step by step: together with W > L2 this makes every
@@ -362,6 +364,7 @@ def main():
     ap.add_argument("--workload", default="decode256", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--tau", type=float, default=None, help="override the workload's threshold")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -85,6 +85,16 @@ __device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
   return r;
 }
+// True in exactly one lane of a converged warp.
+__device__ __forceinline__ bool elect_one() {
+  uint32_t pred;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "elect.sync _|p, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(pred));
+  return pred != 0;
+}
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
@@ -429,7 +439,9 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0 && leader) {
+    // The whole warp walks the schedule and waits on the barriers, so that control flow
+    // and operands stay warp-uniform; one elected lane issues the MMAs and commits.
+    if (leader) {
       int sa = 0, sb = 0;
       uint32_t pa = 0, pb = 0;
       int slab = 0;
@@ -451,12 +463,17 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           const Tile tl = tile_of<kCta>(p, unit, t, 0);
           if (tl.rows == 0) continue;
           const uint32_t idesc = instr_desc(kBlockM * kCta, tl.rows);
-          if (!mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status)) { ok = false; break; }
+          ok = __all_sync(0xffffffffu, mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status));
+          if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * kBlockN;
           for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
-            if (!ra && !mbar_wait(a_full(sa), pa, abort_flag, p.status)) { ok = false; break; }
-            if (!rb && !mbar_wait(b_full(sb), pb, abort_flag, p.status)) { ok = false; break; }
+            if (!__all_sync(0xffffffffu, ra && rb)) {
+              const bool got = mbar_wait(a_full(sa), pa, abort_flag, p.status) &&
+                               mbar_wait(b_full(sb), pb, abort_flag, p.status);
+              ok = __all_sync(0xffffffffu, got);
+              if (!ok) break;
+            }
             tc_fence_after();
             const uint32_t a_lo = a_lo0 + sa * a_step;
             const uint32_t b_lo = b_lo0 + sb * b_step;
@@ -464,16 +481,20 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
             if (++sb == SB) { sb = 0; pb ^= 1u; }
             ra = mbar_test_wait(a_full(sa), pa);
             rb = mbar_test_wait(b_full(sb), pb);
+            if (elect_one()) {
 #pragma unroll
-            for (int k = 0; k < kBlockK / kUmmaK; ++k) {
-              // advancing 16 elements along K inside the swizzle span = +32 bytes = +2 in the address field
-              umma_bf16<kCta>(d_tmem, desc_hi | (a_lo + 2u * k), desc_hi | (b_lo + 2u * k), idesc,
-                              (ks | k) != 0 ? 1u : 0u);
+              for (int k = 0; k < kBlockK / kUmmaK; ++k) {
+                // advancing 16 elements along K inside the swizzle span = +32 bytes = +2 in the address field
+                umma_bf16<kCta>(d_tmem, desc_hi | (a_lo + 2u * k), desc_hi | (b_lo + 2u * k), idesc,
+                                (ks | k) != 0 ? 1u : 0u);
+              }
+              umma_commit<kCta>(released(slab & (kRelease - 1)));   // both slabs are free once these MMAs are done
             }
-            umma_commit<kCta>(released(slab & (kRelease - 1)));   // both slabs are free once these MMAs are done
+            __syncwarp();
           }
           if (!ok) break;
-          umma_commit<kCta>(acc_full(acc));   // accumulator complete (in both CTAs of a pair)
+          if (elect_one()) umma_commit<kCta>(acc_full(acc));   // accumulator complete (in both CTAs of a pair)
+          __syncwarp();
           if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
         }
       }
