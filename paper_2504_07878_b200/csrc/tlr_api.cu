@@ -60,7 +60,7 @@ struct tlr_ctx {
   tlr_path forced = TLR_PATH_AUTO;
   bool tc_ok = false;
   EncodeTiledFn encode = nullptr;
-  CUtensorMap map_w64, map_w16;
+  CUtensorMap map_w128, map_w64, map_w16;
 
   Partial* partials = nullptr;
   unsigned int* ticket = nullptr;
@@ -213,7 +213,7 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
         qres == cudaDriverEntryPointSuccess && fn != nullptr) {
       c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-      if (make_map(c, &c->map_w64, W_bf16_dev, V, d, 64) && make_map(c, &c->map_w16, W_bf16_dev, V, d, 16) &&
+      if (make_map(c, &c->map_w128, W_bf16_dev, V, d, 128) && make_map(c, &c->map_w64, W_bf16_dev, V, d, 64) && make_map(c, &c->map_w16, W_bf16_dev, V, d, 16) &&
           tlr::tc_prepare() == cudaSuccess) {
         c->tc_ok = true;
       }
@@ -299,7 +299,7 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
       p.b_stages = cfg.b_stages;
       p.partials = ctx->partials;
       p.status = ctx->status;
-      e = tlr::launch_tc_projection(map_h, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
+      e = tlr::launch_tc_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
     } else {
       tlr::SimtLaunch a;
       a.W = ctx->W;

@@ -135,8 +135,9 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
       tlr::tc_plan(n, V, cfg.cta, workers_max, kStaticMaxChunks, &tp);
       chunks = tp.chunks;
       const int units = tp.chunks * tp.row_units;
-      CUtensorMap map_h, map_w64, map_w16;
-      if (!encode_map(&map_h, h_bf16_dev, n, d, cfg.a_rows) || !encode_map(&map_w64, W_bf16_dev, V, d, 64) ||
+      CUtensorMap map_h, map_w128, map_w64, map_w16;
+      if (!encode_map(&map_h, h_bf16_dev, n, d, cfg.a_rows) || !encode_map(&map_w128, W_bf16_dev, V, d, 128) ||
+          !encode_map(&map_w64, W_bf16_dev, V, d, 64) ||
           !encode_map(&map_w16, W_bf16_dev, V, d, 16))
         return TLR_ERR_CUDA;
       tlr::TcParams p;
@@ -152,7 +153,7 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
       p.b_stages = cfg.b_stages;
       p.partials = partials;
       p.status = status;
-      if (tlr::launch_tc_projection(map_h, map_w64, map_w16, p, cfg, units < workers_max ? units : workers_max,
+      if (tlr::launch_tc_projection(map_h, map_w128, map_w64, map_w16, p, cfg, units < workers_max ? units : workers_max,
                                     stream) != cudaSuccess)
         return TLR_ERR_CUDA;
     } else {

@@ -313,6 +313,7 @@ __device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int 
 template <int kCta>
 __global__ void __launch_bounds__(kThreads, 1)
 tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
+                     const __grid_constant__ CUtensorMap map_w128,
                      const __grid_constant__ CUtensorMap map_w64,
                      const __grid_constant__ CUtensorMap map_w16,
                      const TcParams p) {
@@ -402,6 +403,8 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
             const uint32_t bar = (kCta == 2) ? map_to_cta(b_full(stage), 0) : b_full(stage);
             if (leader) mbar_expect_tx(b_full(stage), tl.rows * kRowBytes);   // both CTAs' bytes
             int r = 0;
+            for (; my_rows - r >= 128; r += 128)
+              tma_load_2d<kCta>(dst + r * kRowBytes, &map_w128, bar, ks * kBlockK, my_v0 + r);
             for (; my_rows - r >= 64; r += 64)
               tma_load_2d<kCta>(dst + r * kRowBytes, &map_w64, bar, ks * kBlockK, my_v0 + r);
             for (; my_rows - r >= 16; r += 16)
@@ -652,8 +655,9 @@ cudaError_t tc_prepare() {
   return e;
 }
 
-cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w64, const CUtensorMap& map_w16,
-                                 const TcParams& p, const TcConfig& c, int workers, cudaStream_t stream) {
+cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w128, const CUtensorMap& map_w64,
+                                 const CUtensorMap& map_w16, const TcParams& p, const TcConfig& c, int workers,
+                                 cudaStream_t stream) {
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(static_cast<unsigned>(workers * c.cta), 1, 1);
   cfg.blockDim = dim3(kThreads, 1, 1);
@@ -669,10 +673,10 @@ cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& ma
   cfg.attrs = attr;
   if (c.cta == 1) {
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1>, map_h, map_w64, map_w16, p);
+    return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1>, map_h, map_w128, map_w64, map_w16, p);
   }
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2>, map_h, map_w64, map_w16, p);
+  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2>, map_h, map_w128, map_w64, map_w16, p);
 }
 
 }  // namespace tlr

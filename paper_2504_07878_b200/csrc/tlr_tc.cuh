@@ -37,7 +37,8 @@ int tc_threads();
 void tc_configure(int n, TcConfig* c);
 void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan);
 cudaError_t tc_prepare();   // opt in to the kernels' dynamic shared memory size (once per device)
-cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w64, const CUtensorMap& map_w16,
-                                 const TcParams& p, const TcConfig& c, int workers, cudaStream_t stream);
+cudaError_t launch_tc_projection(const CUtensorMap& map_h, const CUtensorMap& map_w128, const CUtensorMap& map_w64,
+                                 const CUtensorMap& map_w16, const TcParams& p, const TcConfig& c, int workers,
+                                 cudaStream_t stream);
 
 }  // namespace tlr
