@@ -172,8 +172,15 @@ def run_ours(args):
     plan = P.tlr_plan_query(routers[0].ctx, n)
     stream = torch.cuda.current_stream()
 
+    variant_args = {}
+    if args.variants:
+        seq_len = args.seq_len if args.seq_len > 0 else (512 if n % 512 == 0 else 1)
+        variant_args = {"tau_per_row": torch.full((n,), tau, dtype=torch.float32, device="cuda"),
+                        "seq_len": seq_len,
+                        "first_routed": torch.zeros(n // seq_len, dtype=torch.int32, device="cuda")}
+
     def step(i):
-        routers[i % copies].route(h_dev, tau, stream)
+        routers[i % copies].route(h_dev, tau, stream, **variant_args)
 
     def barrier():
         if world > 1:
@@ -276,7 +283,9 @@ def run_ours(args):
                    "l2": "inputs larger than L2: W is %.0f MB and two device copies of it alternate between steps"
                          % (2 * V * d / 1e6),
                    "path": int(plan.path), "grid": int(plan.grid), "block": int(plan.block),
-                   "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed},
+                   "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed,
+                   "variants": ("per-row tau + first routed per sequence of %d" % variant_args["seq_len"])
+                   if variant_args else "none"},
         "e2e": {"value": job_throughput(world, n, e2e_s / esteps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)"},
         "gpu_launches": int(plan.launches) * args.steps,
@@ -365,6 +374,10 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--tau", type=float, default=None, help="override the workload's threshold")
+    ap.add_argument("--variants", action="store_true",
+                    help="route with per-row thresholds and report the first routed position per sequence "
+                         "(tlr_route_ex; sequences of --seq-len rows)")
+    ap.add_argument("--seq-len", type=int, default=0)
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

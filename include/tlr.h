@@ -116,6 +116,38 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
                      int32_t* routed_count_dev, void* cuda_stream);
 
 /*
+ * tlr_route_ex -- tlr_route with the routing variants the paper's Sec. 2 and Sec. 3 name.
+ *   opt->tau_per_row_dev   optional float [n] on the device: row i is compared with
+ *                          tau_per_row_dev[i] instead of the scalar tau (the threshold is a
+ *                          per-user setting in the paper's front end, Sec. 3.1, so a batch of
+ *                          sessions carries one threshold per row).  NULL = scalar tau.
+ *   opt->route_above       0: route iff score < tau (Sec. 3.1).  1: route iff score > tau, the
+ *                          polarity of the deferral rule of Sec. 2.2 (defer when the deferral
+ *                          probability exceeds eta).  A row whose score is not a number is
+ *                          routed under either polarity.
+ *   opt->seq_len,          when seq_len > 0 the n rows are n / seq_len sequences of seq_len
+ *   opt->first_routed_dev  consecutive positions (n must be a multiple of seq_len) and
+ *                          first_routed_dev (int32 [n / seq_len], device) receives, per
+ *                          sequence, the position within the sequence of its first routed row,
+ *                          or seq_len if none is routed: after the large model has supplied a
+ *                          token the small model re-processes the whole context (Sec. 4.1, the
+ *                          multi-round prefill of Sec. 3), and this is where it has to stop next.
+ * opt == NULL behaves exactly like tlr_route.  Same outputs, stream semantics and errors as
+ * tlr_route; TLR_ERR_ARG also for seq_len > 0 with n % seq_len != 0 or a NULL first_routed_dev.
+ */
+typedef struct {
+  const float* tau_per_row_dev;
+  int32_t route_above;
+  int32_t seq_len;
+  int32_t* first_routed_dev;
+} tlr_route_options;
+
+tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
+                        const tlr_route_options* opt, int32_t* token_dev, float* conf_dev,
+                        float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev,
+                        int32_t* routed_count_dev, void* cuda_stream);
+
+/*
  * tlr_route_host -- the same step with HOST buffers: copies h to the device, runs
  * tlr_route, copies the six results back, and synchronises the stream before
  * returning.  Host buffers may be pageable or pinned (pinned is faster).  Output

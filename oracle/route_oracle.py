@@ -19,6 +19,9 @@ What it computes, per decoding position i (one row of ``h``):
      below" the threshold, Sec. 3.1; Sec. 2.1: routing scores against a
      predefined threshold tau)
   6. routed_idx = ascending positions with route set; routed_count = how many
+  Variants of steps 5-6: one threshold per row, the opposite polarity (Sec. 2.2:
+  defer when the score exceeds the threshold), and the first routed position of
+  every sequence (Sec. 4.1: where the re-processing of a returned context stops).
 
 All arithmetic is fp64 on the exact values of the bf16 inputs.  The only
 library primitive used as a step is the dense matrix product of step 1.  Rows
@@ -92,17 +95,41 @@ def row_statistics(z: np.ndarray):
     return token.astype(np.int32), conf, entropy, gap
 
 
-def route_decision(conf: np.ndarray, tau: float):
+def route_decision(conf: np.ndarray, tau, route_above: bool = False):
     """Steps 5-6.  ``tau`` is rounded to fp32 first: that is the value the C-ABI carries.
 
-    A row whose confidence is not a number is routed (fail-safe to the large
-    model): the test is "not (conf >= tau)", which equals "conf < tau" for
-    every finite confidence.
+    ``tau`` is a scalar or one threshold per row (the threshold is a per-user
+    setting in the front end, Sec. 3.1).  ``route_above`` switches to the
+    polarity of the deferral rule of Sec. 2.2 (defer when the score exceeds
+    the threshold).  A row whose confidence is not a number is routed under
+    either polarity (fail-safe to the large model): the tests are
+    "not (conf >= tau)" and "not (conf <= tau)", which equal "conf < tau" and
+    "conf > tau" for every finite confidence.
     """
-    tau32 = float(np.float32(tau))
-    mask = np.logical_not(conf >= tau32).astype(np.uint8)
+    tau32 = np.asarray(tau, dtype=np.float32).astype(np.float64)
+    if route_above:
+        mask = np.logical_not(conf <= tau32).astype(np.uint8)
+    else:
+        mask = np.logical_not(conf >= tau32).astype(np.uint8)
     idx = np.flatnonzero(mask).astype(np.int32)
-    return mask, idx, int(idx.size), tau32
+    return mask, idx, int(idx.size), (float(tau32) if tau32.ndim == 0 else tau32)
+
+
+def first_routed(route_mask: np.ndarray, seq_len: int) -> np.ndarray:
+    """Per sequence of ``seq_len`` consecutive rows: position of its first routed row, or seq_len.
+
+    After the large model has supplied a token the small model re-processes the whole
+    context (Sec. 4.1; the multi-round prefill of Sec. 3): this is where it stops next.
+    """
+    n = route_mask.shape[0]
+    if seq_len <= 0 or n % seq_len != 0:
+        raise ValueError("n must be a positive multiple of seq_len")
+    out = np.full(n // seq_len, seq_len, dtype=np.int32)
+    for b in range(n // seq_len):
+        hits = np.flatnonzero(route_mask[b * seq_len:(b + 1) * seq_len])
+        if hits.size:
+            out[b] = hits[0]
+    return out
 
 
 def route_oracle(h_bits: np.ndarray, W_bits: np.ndarray, tau: float,
@@ -128,9 +155,9 @@ def route_oracle(h_bits: np.ndarray, W_bits: np.ndarray, tau: float,
     return RouteResult(token, conf, entropy, mask, idx, count, gap, tau32)
 
 
-def with_threshold(result: RouteResult, tau: float) -> RouteResult:
-    """The same per-row scores with steps 5-6 redone for another threshold."""
-    mask, idx, count, tau32 = route_decision(result.conf, tau)
+def with_threshold(result: RouteResult, tau, route_above: bool = False) -> RouteResult:
+    """The same per-row scores with steps 5-6 redone for another threshold or polarity."""
+    mask, idx, count, tau32 = route_decision(result.conf, tau, route_above)
     return RouteResult(result.token, result.conf, result.entropy, mask, idx, count, result.top2_gap, tau32)
 
 

@@ -28,6 +28,11 @@ class TlrPlan(ctypes.Structure):
                 ("vocab_chunks", c_int32), ("smem_bytes", c_int32), ("launches", c_int32), ("reserved", c_int32)]
 
 
+class TlrRouteOptions(ctypes.Structure):
+    _fields_ = [("tau_per_row_dev", c_void_p), ("route_above", c_int32), ("seq_len", c_int32),
+                ("first_routed_dev", c_void_p)]
+
+
 class TlrError(RuntimeError):
     def __init__(self, code: int, where: str):
         self.code = code
@@ -49,6 +54,8 @@ def load_library() -> ctypes.CDLL:
     P = c_void_p
     lib.tlr_create.argtypes = [c_int32, c_int32, P, c_int32, POINTER(P)]
     lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_route_ex.argtypes = [P, P, c_int32, c_float, POINTER(TlrRouteOptions), P, P, P, P, P, P, P]
+    lib.tlr_route_ex.restype = c_int32
     lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_destroy.argtypes = [P]
     lib.tlr_status_string.argtypes = [c_int32]
@@ -103,6 +110,15 @@ def tlr_route(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, rout
     """All tensor arguments are CUDA tensors (or raw device addresses).  Asynchronous on `stream`."""
     _check(load_library().tlr_route(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy), _ptr(route_mask),
                                     _ptr(routed_idx), _ptr(routed_count), _stream_handle(stream)), "tlr_route")
+
+
+def tlr_route_ex(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count, stream=None,
+                 tau_per_row=None, route_above: bool = False, seq_len: int = 0, first_routed=None):
+    """tlr_route with per-row thresholds, the opposite polarity, and the first routed position per sequence."""
+    opt = TlrRouteOptions(_ptr(tau_per_row), 1 if route_above else 0, int(seq_len), _ptr(first_routed))
+    _check(load_library().tlr_route_ex(ctx, _ptr(h), n, tau, byref(opt), _ptr(token), _ptr(conf), _ptr(entropy),
+                                       _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
+                                       _stream_handle(stream)), "tlr_route_ex")
 
 
 def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count,
@@ -175,14 +191,20 @@ class Router:
             self.routed_idx = torch.empty(max_n, dtype=torch.int32, device=dev)
             self.routed_count = torch.zeros(1, dtype=torch.int32, device=dev)
 
-    def route(self, h: torch.Tensor, tau: float, stream=None):
+    def route(self, h: torch.Tensor, tau: float, stream=None, tau_per_row=None, route_above=False, seq_len=0,
+              first_routed=None):
         """Enqueues one routing step; returns views of the output tensors (valid after the stream syncs)."""
         if not (h.is_cuda and h.dtype == torch.bfloat16 and h.dim() == 2 and h.is_contiguous()
                 and h.shape[1] == self.d):
             raise ValueError("h must be a contiguous CUDA bf16 [n, d] tensor")
         n = h.shape[0]
-        tlr_route(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
-                  self.routed_count, stream)
+        if tau_per_row is None and not route_above and seq_len == 0:
+            tlr_route(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
+                      self.routed_count, stream)
+        else:
+            tlr_route_ex(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
+                         self.routed_count, stream, tau_per_row=tau_per_row, route_above=route_above,
+                         seq_len=seq_len, first_routed=first_routed)
         return (self.token[:n], self.conf[:n], self.entropy[:n], self.route_mask[:n], self.routed_idx,
                 self.routed_count)
 

@@ -252,7 +252,17 @@ tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out) {
 tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, int32_t* token_dev, float* conf_dev,
                      float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev, int32_t* routed_count_dev,
                      void* cuda_stream) {
+  return tlr_route_ex(ctx, h_bf16_dev, n, tau, nullptr, token_dev, conf_dev, entropy_dev, route_mask_dev,
+                      routed_idx_dev, routed_count_dev, cuda_stream);
+}
+
+tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, const tlr_route_options* opt,
+                        int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
+                        int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream) {
   if (ctx == nullptr || n < 0 || routed_count_dev == nullptr) return TLR_ERR_ARG;
+  if (opt != nullptr && opt->seq_len > 0 && (n % opt->seq_len != 0 || opt->first_routed_dev == nullptr))
+    return TLR_ERR_ARG;
+  if (opt != nullptr && opt->seq_len < 0) return TLR_ERR_ARG;
   if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
   if (n > 0) {
     if (h_bf16_dev == nullptr || token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr ||
@@ -323,6 +333,10 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
   f.n = n;
   f.chunks = plan.vocab_chunks;
   f.tau = tau;
+  f.tau_rows = opt != nullptr ? opt->tau_per_row_dev : nullptr;
+  f.route_above = (opt != nullptr && opt->route_above != 0) ? 1 : 0;
+  f.seq_len = opt != nullptr ? opt->seq_len : 0;
+  f.first_routed = opt != nullptr ? opt->first_routed_dev : nullptr;
   f.token = token_dev;
   f.conf = conf_dev;
   f.entropy = entropy_dev;

@@ -92,6 +92,10 @@ struct FinishLaunch {
   const Partial* partials;  // [n][chunks]
   int n, chunks;
   float tau;
+  const float* tau_rows;    // optional per-row thresholds [n]
+  int route_above;          // 0: route iff conf < tau; 1: route iff conf > tau
+  int seq_len;              // > 0: also report the first routed position of every sequence
+  int32_t* first_routed;    // [n / seq_len] when seq_len > 0
   int32_t* token;
   float* conf;
   float* entropy;

@@ -90,13 +90,27 @@ __device__ __forceinline__ int score_row(const Partial& acc, const FinishLaunch&
     ent = conf;
     atomicOr(a.status, TLR_DEV_NONFINITE);
   }
-  // "not (conf >= tau)": equals conf < tau for numbers, and routes a NaN row.
-  const int flag = (conf >= a.tau) ? 0 : 1;
+  // "not (conf >= tau)": equals conf < tau for numbers, and routes a NaN row; likewise
+  // "not (conf <= tau)" for the opposite polarity.
+  const float tau = a.tau_rows != nullptr ? a.tau_rows[row] : a.tau;
+  const int flag = a.route_above ? ((conf <= tau) ? 0 : 1) : ((conf >= tau) ? 0 : 1);
   a.token[row] = acc.idx;
   a.conf[row] = conf;
   a.entropy[row] = ent;
   a.route_mask[row] = static_cast<uint8_t>(flag);
   return flag;
+}
+
+// First routed position of every sequence: an atomic minimum per sequence over the
+// routed rows.  Called by the one block that compacts, before (init) and during the pass.
+__device__ __forceinline__ void first_routed_init(const FinishLaunch& a) {
+  if (a.seq_len > 0) {
+    for (int b = threadIdx.x; b < a.n / a.seq_len; b += blockDim.x) a.first_routed[b] = a.seq_len;
+    __syncthreads();
+  }
+}
+__device__ __forceinline__ void first_routed_note(const FinishLaunch& a, int row) {
+  if (a.seq_len > 0) atomicMin(a.first_routed + row / a.seq_len, row % a.seq_len);
 }
 
 // Programmatic dependent launch: let the next kernel in the stream be scheduled now (it
@@ -220,6 +234,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   }
   if (blockIdx.x != 0) return;
+  first_routed_init(a);
   const int i = threadIdx.x;
   int flag = 0;
   if (i < a.n) flag = single_block ? static_cast<int>(flags[i]) : static_cast<int>(__ldcg(a.route_mask + i));
@@ -233,7 +248,10 @@ finish_small_kernel(const FinishLaunch a, const int L) {
     before += (w < warp) ? c : 0;
     total += c;
   }
-  if (flag) a.routed_idx[before + __popc(bal & ((1u << lane) - 1u))] = i;
+  if (flag) {
+    a.routed_idx[before + __popc(bal & ((1u << lane) - 1u))] = i;
+    first_routed_note(a, i);
+  }
   if (threadIdx.x == 0) *a.routed_count = total;
 }
 
@@ -263,6 +281,7 @@ finish_kernel(const FinishLaunch a) {
   __threadfence();
 
   // ---- ordered compaction by the last block
+  first_routed_init(a);
   int base_out = 0;
   for (int base = 0; base < a.n; base += kFinishThreads) {
     const int i = base + threadIdx.x;
@@ -277,7 +296,10 @@ finish_kernel(const FinishLaunch a) {
       before += (w < warp) ? c : 0;
       total += c;
     }
-    if (flag) a.routed_idx[base_out + before + __popc(bal & ((1u << lane) - 1u))] = i;
+    if (flag) {
+      a.routed_idx[base_out + before + __popc(bal & ((1u << lane) - 1u))] = i;
+      first_routed_note(a, i);
+    }
     base_out += total;
     __syncthreads();
   }

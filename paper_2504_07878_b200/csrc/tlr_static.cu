@@ -176,6 +176,10 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
   f.n = n;
   f.chunks = chunks;
   f.tau = tau;
+  f.tau_rows = nullptr;
+  f.route_above = 0;
+  f.seq_len = 0;
+  f.first_routed = nullptr;
   f.token = token_dev;
   f.conf = conf_dev;
   f.entropy = entropy_dev;

@@ -270,3 +270,37 @@ def test_generators_are_seeded_and_independent_of_n():
     h1 = S.make_h(4, 8, seed=0).h; h2 = S.make_h(4, 8, seed=0).h
     assert torch.equal(h1, h2)
     assert S.make_h(0, 8).h.shape == (0, 8)
+
+
+# ---------------------------------------------------------------- variants of the decision
+def test_polarity_and_per_row_threshold():
+    conf = np.array([0.1, 0.5, 0.5000001, 0.9, np.nan])
+    below = O.route_decision(conf, 0.5)[0]
+    above = O.route_decision(conf, 0.5, route_above=True)[0]
+    assert below.tolist() == [1, 0, 0, 0, 1]         # strict: 0.5 is not below 0.5; NaN is routed
+    assert above.tolist() == [0, 0, 1, 1, 1]         # strict: 0.5 is not above 0.5; NaN is routed
+    # away from equality and NaN the two polarities are complements
+    hb, Wb = _random_case(n=50, seed=4)
+    r = O.route_oracle(hb, Wb, 0.2)
+    up = O.with_threshold(r, 0.2, route_above=True)
+    assert np.array_equal(up.route_mask, 1 - r.route_mask)
+    # a constant vector is the scalar; a vector applies row by row
+    vec = O.route_decision(conf[:4], np.array([0.05, 0.6, 0.4, 0.95]))[0]
+    assert vec.tolist() == [0, 1, 0, 1]
+    assert np.array_equal(O.route_decision(r.conf, np.full(50, 0.2))[0], r.route_mask)
+
+
+def test_first_routed_position_per_sequence():
+    mask = np.array([0, 0, 1, 1,   0, 0, 0, 0,   1, 0, 0, 1,   0, 0, 0, 1], dtype=np.uint8)
+    assert O.first_routed(mask, 4).tolist() == [2, 4, 0, 3]         # worked by hand; 4 = none routed
+    assert O.first_routed(mask, 16).tolist() == [2]
+    assert O.first_routed(mask, 1).tolist() == (1 - mask).tolist()  # length-1 sequences: 0 if routed else 1
+    # equals the minimum of the segment's entries of the compacted index list
+    rng = np.random.default_rng(3)
+    m = (rng.random(60) < 0.1).astype(np.uint8)
+    idx = np.flatnonzero(m)
+    for b, f in enumerate(O.first_routed(m, 12)):
+        seg = idx[(idx >= 12 * b) & (idx < 12 * (b + 1))]
+        assert f == (seg.min() - 12 * b if seg.size else 12)
+    with pytest.raises(ValueError):
+        O.first_routed(mask, 5)
