@@ -179,6 +179,15 @@ def run_ours(args):
                         "seq_len": seq_len,
                         "first_routed": torch.zeros(n // seq_len, dtype=torch.int32, device="cuda")}
 
+    if args.mlp > 0:
+        g = torch.Generator().manual_seed(0)
+        W1 = (torch.randn(args.mlp, d, generator=g) / d ** 0.5).to(torch.bfloat16).cuda()
+        b1 = (torch.randn(args.mlp, generator=g) * 0.1).cuda()
+        w2 = (torch.randn(args.mlp, generator=g) * 0.5).cuda()
+        for r in routers:
+            r.set_router_mlp(W1, b1, w2, 0.0)
+        variant_args["score_source"] = P.TLR_SCORE_MLP
+
     def step(i):
         routers[i % copies].route(h_dev, tau, stream, **variant_args)
 
@@ -284,11 +293,12 @@ def run_ours(args):
                          % (2 * V * d / 1e6),
                    "path": int(plan.path), "grid": int(plan.grid), "block": int(plan.block),
                    "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed,
-                   "variants": ("per-row tau + first routed per sequence of %d" % variant_args["seq_len"])
-                   if variant_args else "none"},
+                   "variants": (("per-row tau + first routed per sequence of %d" % variant_args["seq_len"])
+                                if "seq_len" in variant_args else "none") +
+                               ("; learned router, hidden width %d" % args.mlp if args.mlp > 0 else "")},
         "e2e": {"value": job_throughput(world, n, e2e_s / esteps), "unit": UNIT, "h2d_bytes_per_step": h2d,
                 "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)"},
-        "gpu_launches": int(plan.launches) * args.steps,
+        "gpu_launches": (int(plan.launches) + (1 if args.mlp > 0 else 0)) * args.steps,
         "clocks": sampler.summary(),
         "roofline": roof,
     }
@@ -378,6 +388,8 @@ def main():
                     help="route with per-row thresholds and report the first routed position per sequence "
                          "(tlr_route_ex; sequences of --seq-len rows)")
     ap.add_argument("--seq-len", type=int, default=0)
+    ap.add_argument("--mlp", type=int, default=0,
+                    help="attach a learned router of this hidden width (random weights) and route on its score")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3

@@ -125,6 +125,8 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
  *                          polarity of the deferral rule of Sec. 2.2 (defer when the deferral
  *                          probability exceeds eta).  A row whose score is not a number is
  *                          routed under either polarity.
+ *   opt->score_source,     which score decides (see tlr_set_router_mlp below); mlp_score_dev optionally
+ *   opt->mlp_score_dev     receives the learned score of every row.
  *   opt->seq_len,          when seq_len > 0 the n rows are n / seq_len sequences of seq_len
  *   opt->first_routed_dev  consecutive positions (n must be a multiple of seq_len) and
  *                          first_routed_dev (int32 [n / seq_len], device) receives, per
@@ -140,7 +142,29 @@ typedef struct {
   int32_t route_above;
   int32_t seq_len;
   int32_t* first_routed_dev;
+  int32_t score_source;      /* TLR_SCORE_CONF (0) or TLR_SCORE_MLP (1): which score is compared with tau */
+  float* mlp_score_dev;      /* optional float [n] out: the learned score of every row (needs tlr_set_router_mlp) */
 } tlr_route_options;
+
+#define TLR_SCORE_CONF 0   /* the small model's max softmax probability (default) */
+#define TLR_SCORE_MLP 1    /* the learned score of tlr_set_router_mlp */
+
+/*
+ * tlr_set_router_mlp -- attach a learned router to the context.  The paper's deployed score is
+ * "an MLP classifier which operates on the last-layer hidden state" (Sec. 3.1, Sec. 2.1) whose
+ * width, activation and weights it does not give; the shape here is this library's assumption:
+ *     score(h) = sigmoid( w2 . relu(W1 h + b1) + b2 )        in (0, 1), high = keep the small model
+ *   d_hidden        hidden width, > 0
+ *   W1_bf16_dev     bf16 [d_hidden, d] row-major on the device;  b1_dev, w2_dev  float [d_hidden];  b2 scalar
+ * The pointers are BORROWED for the life of the context (or until replaced by another call).
+ * Allocates ceil(d_hidden / 32) floats per max_n row for partial sums.  With a router attached, tlr_route_ex computes
+ * the learned score of every row in one extra small kernel when opt->score_source == TLR_SCORE_MLP
+ * or opt->mlp_score_dev != NULL; token, conf and entropy are produced as always.
+ * Errors: TLR_ERR_ARG, TLR_ERR_NOMEM.  tlr_route_ex returns TLR_ERR_ARG when the learned score is
+ * requested but no router is attached.
+ */
+tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf16_dev, const float* b1_dev,
+                              const float* w2_dev, float b2);
 
 tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
                         const tlr_route_options* opt, int32_t* token_dev, float* conf_dev,

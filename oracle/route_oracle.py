@@ -34,7 +34,9 @@ vectors, an independent library softmax/entropy, a pure-Python brute force,
 threshold invariants (tau=0, tau=1, monotone count -- Table 1 "Routing
 Number"), and distributional closed forms of the synthetic workload.
 Parity unpinned: anything tied to the paper's dataset or trained router
-(accuracy and routed-ratio curves, Figs. 7-8) -- neither is available.
+(accuracy and routed-ratio curves, Figs. 7-8) -- neither is available; and
+mlp_router_score, whose shape the paper does not give (pinned by closed forms
+and a library cross-check only).
 """
 from __future__ import annotations
 
@@ -159,6 +161,24 @@ def with_threshold(result: RouteResult, tau, route_above: bool = False) -> Route
     """The same per-row scores with steps 5-6 redone for another threshold or polarity."""
     mask, idx, count, tau32 = route_decision(result.conf, tau, route_above)
     return RouteResult(result.token, result.conf, result.entropy, mask, idx, count, result.top2_gap, tau32)
+
+
+def mlp_router_score(h_bits: np.ndarray, W1_bits: np.ndarray, b1, w2, b2: float) -> np.ndarray:
+    """Learned routing score sigmoid(w2 . relu(W1 h + b1) + b2), fp64, one value per row.
+
+    The paper routes on "an MLP classifier which operates on the last-layer hidden
+    state" (Sec. 3.1; Sec. 2.1) without giving its shape; one hidden layer with ReLU
+    and a sigmoid output is this repository's assumption, so this function is pinned
+    only by mathematics (closed forms, a library cross-check), not by the paper:
+    parity unpinned by the paper.  W1 is bf16 bits [d_hidden, d]; b1, w2 are fp32.
+    """
+    h64 = bf16_bits_to_f64(h_bits)
+    W1 = bf16_bits_to_f64(W1_bits)
+    b1 = np.asarray(b1, dtype=np.float32).astype(np.float64)
+    w2 = np.asarray(w2, dtype=np.float32).astype(np.float64)
+    hidden = np.maximum(h64 @ W1.T + b1[None, :], 0.0)
+    logit = hidden @ w2 + float(np.float32(b2))
+    return 1.0 / (1.0 + np.exp(-logit))
 
 
 def percentile_tau(conf: np.ndarray, fraction: float = 0.07) -> float:

@@ -21,6 +21,7 @@ TLR_ERR_NOMEM, TLR_ERR_TOO_MANY_ROWS, TLR_ERR_DEVICE_STATUS = 5, 6, 7
 TLR_PATH_AUTO, TLR_PATH_SIMT, TLR_PATH_TC = 0, 1, 2
 TLR_DEV_WAIT_TIMEOUT, TLR_DEV_NONFINITE = 1, 2
 TLR_STATIC_MAX_ROWS = 1024
+TLR_SCORE_CONF, TLR_SCORE_MLP = 0, 1
 
 
 class TlrPlan(ctypes.Structure):
@@ -30,7 +31,7 @@ class TlrPlan(ctypes.Structure):
 
 class TlrRouteOptions(ctypes.Structure):
     _fields_ = [("tau_per_row_dev", c_void_p), ("route_above", c_int32), ("seq_len", c_int32),
-                ("first_routed_dev", c_void_p)]
+                ("first_routed_dev", c_void_p), ("score_source", c_int32), ("mlp_score_dev", c_void_p)]
 
 
 class TlrError(RuntimeError):
@@ -56,6 +57,8 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_route_ex.argtypes = [P, P, c_int32, c_float, POINTER(TlrRouteOptions), P, P, P, P, P, P, P]
     lib.tlr_route_ex.restype = c_int32
+    lib.tlr_set_router_mlp.argtypes = [P, c_int32, P, P, P, c_float]
+    lib.tlr_set_router_mlp.restype = c_int32
     lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_destroy.argtypes = [P]
     lib.tlr_status_string.argtypes = [c_int32]
@@ -113,12 +116,20 @@ def tlr_route(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, rout
 
 
 def tlr_route_ex(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count, stream=None,
-                 tau_per_row=None, route_above: bool = False, seq_len: int = 0, first_routed=None):
-    """tlr_route with per-row thresholds, the opposite polarity, and the first routed position per sequence."""
-    opt = TlrRouteOptions(_ptr(tau_per_row), 1 if route_above else 0, int(seq_len), _ptr(first_routed))
+                 tau_per_row=None, route_above: bool = False, seq_len: int = 0, first_routed=None,
+                 score_source: int = 0, mlp_score=None):
+    """tlr_route with per-row thresholds, the opposite polarity, the first routed position per sequence,
+    and the learned router score (score_source=TLR_SCORE_MLP after tlr_set_router_mlp)."""
+    opt = TlrRouteOptions(_ptr(tau_per_row), 1 if route_above else 0, int(seq_len), _ptr(first_routed),
+                          int(score_source), _ptr(mlp_score))
     _check(load_library().tlr_route_ex(ctx, _ptr(h), n, tau, byref(opt), _ptr(token), _ptr(conf), _ptr(entropy),
                                        _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
                                        _stream_handle(stream)), "tlr_route_ex")
+
+
+def tlr_set_router_mlp(ctx, d_hidden: int, W1, b1, w2, b2: float):
+    """Attach score(h) = sigmoid(w2 . relu(W1 h + b1) + b2); W1 bf16 [d_hidden, d], b1/w2 float [d_hidden] (CUDA)."""
+    _check(load_library().tlr_set_router_mlp(ctx, d_hidden, _ptr(W1), _ptr(b1), _ptr(w2), b2), "tlr_set_router_mlp")
 
 
 def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count,
@@ -191,20 +202,26 @@ class Router:
             self.routed_idx = torch.empty(max_n, dtype=torch.int32, device=dev)
             self.routed_count = torch.zeros(1, dtype=torch.int32, device=dev)
 
+    def set_router_mlp(self, W1: torch.Tensor, b1: torch.Tensor, w2: torch.Tensor, b2: float):
+        """Attach a learned router; the tensors are kept alive by this object."""
+        self._mlp = (W1, b1, w2)
+        tlr_set_router_mlp(self.ctx, W1.shape[0], W1, b1, w2, float(b2))
+
     def route(self, h: torch.Tensor, tau: float, stream=None, tau_per_row=None, route_above=False, seq_len=0,
-              first_routed=None):
+              first_routed=None, score_source=0, mlp_score=None):
         """Enqueues one routing step; returns views of the output tensors (valid after the stream syncs)."""
         if not (h.is_cuda and h.dtype == torch.bfloat16 and h.dim() == 2 and h.is_contiguous()
                 and h.shape[1] == self.d):
             raise ValueError("h must be a contiguous CUDA bf16 [n, d] tensor")
         n = h.shape[0]
-        if tau_per_row is None and not route_above and seq_len == 0:
+        if tau_per_row is None and not route_above and seq_len == 0 and score_source == 0 and mlp_score is None:
             tlr_route(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
                       self.routed_count, stream)
         else:
             tlr_route_ex(self.ctx, h, n, tau, self.token, self.conf, self.entropy, self.route_mask, self.routed_idx,
                          self.routed_count, stream, tau_per_row=tau_per_row, route_above=route_above,
-                         seq_len=seq_len, first_routed=first_routed)
+                         seq_len=seq_len, first_routed=first_routed, score_source=score_source,
+                         mlp_score=mlp_score)
         return (self.token[:n], self.conf[:n], self.entropy[:n], self.route_mask[:n], self.routed_idx,
                 self.routed_count)
 

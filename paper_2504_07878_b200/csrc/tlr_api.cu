@@ -75,6 +75,15 @@ struct tlr_ctx {
   int32_t* idx_stage = nullptr;
   int32_t* count_stage = nullptr;
 
+  // learned router (tlr_set_router_mlp)
+  int mlp_hidden = 0;
+  const void* mlp_W1 = nullptr;
+  const float* mlp_b1 = nullptr;
+  const float* mlp_w2 = nullptr;
+  float mlp_b2 = 0.f;
+  float* mlp_scores = nullptr;     // [max_n][hidden blocks] partial sums of the output layer
+  int mlp_blocks_cap = 0;
+
   bool timing = false;
   std::vector<cudaEvent_t> events;   // pairs, created lazily
   int timed = 0;
@@ -138,6 +147,7 @@ void free_all(tlr_ctx* c) {
   cudaFree(c->mask_stage);
   cudaFree(c->idx_stage);
   cudaFree(c->count_stage);
+  cudaFree(c->mlp_scores);
   for (cudaEvent_t e : c->events) cudaEventDestroy(e);
   delete c;
 }
@@ -234,6 +244,29 @@ tlr_status tlr_destroy(tlr_ctx* ctx) {
   return TLR_OK;
 }
 
+tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf16_dev, const float* b1_dev,
+                              const float* w2_dev, float b2) {
+  if (ctx == nullptr || d_hidden <= 0 || W1_bf16_dev == nullptr || b1_dev == nullptr || w2_dev == nullptr)
+    return TLR_ERR_ARG;
+  const int blocks = tlr::mlp_hidden_blocks(d_hidden);
+  if (ctx->mlp_scores == nullptr || blocks > ctx->mlp_blocks_cap) {
+    cudaFree(ctx->mlp_scores);
+    ctx->mlp_scores = nullptr;
+    if (cudaMalloc(&ctx->mlp_scores, static_cast<size_t>(ctx->max_n) * blocks * sizeof(float)) != cudaSuccess) {
+      cudaGetLastError();
+      ctx->mlp_hidden = 0;
+      return TLR_ERR_NOMEM;
+    }
+    ctx->mlp_blocks_cap = blocks;
+  }
+  ctx->mlp_hidden = d_hidden;
+  ctx->mlp_W1 = W1_bf16_dev;
+  ctx->mlp_b1 = b1_dev;
+  ctx->mlp_w2 = w2_dev;
+  ctx->mlp_b2 = b2;
+  return TLR_OK;
+}
+
 tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path) {
   if (ctx == nullptr) return TLR_ERR_ARG;
   if (path != TLR_PATH_AUTO && path != TLR_PATH_SIMT && path != TLR_PATH_TC) return TLR_ERR_ARG;
@@ -263,6 +296,9 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
   if (opt != nullptr && opt->seq_len > 0 && (n % opt->seq_len != 0 || opt->first_routed_dev == nullptr))
     return TLR_ERR_ARG;
   if (opt != nullptr && opt->seq_len < 0) return TLR_ERR_ARG;
+  const bool want_mlp = opt != nullptr && (opt->score_source == TLR_SCORE_MLP || opt->mlp_score_dev != nullptr);
+  if (opt != nullptr && opt->score_source != TLR_SCORE_CONF && opt->score_source != TLR_SCORE_MLP) return TLR_ERR_ARG;
+  if (want_mlp && ctx->mlp_hidden == 0) return TLR_ERR_ARG;
   if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
   if (n > 0) {
     if (h_bf16_dev == nullptr || token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr ||
@@ -328,11 +364,30 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
     }
   }
 
+  if (want_mlp && n > 0) {
+    tlr::MlpLaunch m;
+    m.h = h_bf16_dev;
+    m.W1 = ctx->mlp_W1;
+    m.b1 = ctx->mlp_b1;
+    m.w2 = ctx->mlp_w2;
+    m.b2 = ctx->mlp_b2;
+    m.n = n;
+    m.d = ctx->d;
+    m.d_hidden = ctx->mlp_hidden;
+    m.partial = ctx->mlp_scores;
+    if (tlr::launch_mlp_score(m, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  }
+
   tlr::FinishLaunch f;
   f.partials = ctx->partials;
   f.n = n;
   f.chunks = plan.vocab_chunks;
   f.tau = tau;
+  f.mlp_partial = want_mlp ? ctx->mlp_scores : nullptr;
+  f.mlp_blocks = want_mlp ? tlr::mlp_hidden_blocks(ctx->mlp_hidden) : 0;
+  f.mlp_b2 = ctx->mlp_b2;
+  f.decide_on_mlp = (opt != nullptr && opt->score_source == TLR_SCORE_MLP) ? 1 : 0;
+  f.mlp_score_out = opt != nullptr ? opt->mlp_score_dev : nullptr;
   f.tau_rows = opt != nullptr ? opt->tau_per_row_dev : nullptr;
   f.route_above = (opt != nullptr && opt->route_above != 0) ? 1 : 0;
   f.seq_len = opt != nullptr ? opt->seq_len : 0;

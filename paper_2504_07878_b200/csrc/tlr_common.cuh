@@ -92,6 +92,11 @@ struct FinishLaunch {
   const Partial* partials;  // [n][chunks]
   int n, chunks;
   float tau;
+  const float* mlp_partial;   // optional [n][mlp_blocks]: partial sums of the learned router's output layer
+  int mlp_blocks;
+  float mlp_b2;
+  int decide_on_mlp;          // 1: the learned score is compared with tau instead of conf
+  float* mlp_score_out;       // optional [n]: the learned score
   const float* tau_rows;    // optional per-row thresholds [n]
   int route_above;          // 0: route iff conf < tau; 1: route iff conf > tau
   int seq_len;              // > 0: also report the first routed position of every sequence
@@ -106,5 +111,17 @@ struct FinishLaunch {
   uint32_t* status;
 };
 cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
+
+struct MlpLaunch {
+  const void* h;        // bf16 [n][d]
+  const void* W1;       // bf16 [d_hidden][d]
+  const float* b1;      // [d_hidden]
+  const float* w2;      // [d_hidden]
+  float b2;
+  int n, d, d_hidden;
+  float* partial;       // [n][mlp_hidden_blocks(d_hidden)] out
+};
+int mlp_hidden_blocks(int d_hidden);
+cudaError_t launch_mlp_score(const MlpLaunch& a, cudaStream_t stream);
 
 }  // namespace tlr

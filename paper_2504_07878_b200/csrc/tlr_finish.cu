@@ -93,7 +93,16 @@ __device__ __forceinline__ int score_row(const Partial& acc, const FinishLaunch&
   // "not (conf >= tau)": equals conf < tau for numbers, and routes a NaN row; likewise
   // "not (conf <= tau)" for the opposite polarity.
   const float tau = a.tau_rows != nullptr ? a.tau_rows[row] : a.tau;
-  const int flag = a.route_above ? ((conf <= tau) ? 0 : 1) : ((conf >= tau) ? 0 : 1);
+  float score = conf;
+  if (a.mlp_partial != nullptr) {
+    // learned score: the output layer's partial sums in a fixed order, then the sigmoid
+    float v = a.mlp_b2;
+    for (int b = 0; b < a.mlp_blocks; ++b) v += __ldcg(a.mlp_partial + static_cast<size_t>(row) * a.mlp_blocks + b);
+    const float learned = 1.0f / (1.0f + expf(-v));
+    if (a.mlp_score_out != nullptr) a.mlp_score_out[row] = learned;
+    if (a.decide_on_mlp) score = learned;
+  }
+  const int flag = a.route_above ? ((score <= tau) ? 0 : 1) : ((score >= tau) ? 0 : 1);
   a.token[row] = acc.idx;
   a.conf[row] = conf;
   a.entropy[row] = ent;

@@ -176,6 +176,11 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
   f.n = n;
   f.chunks = chunks;
   f.tau = tau;
+  f.mlp_partial = nullptr;
+  f.mlp_blocks = 0;
+  f.mlp_b2 = 0.f;
+  f.decide_on_mlp = 0;
+  f.mlp_score_out = nullptr;
   f.tau_rows = nullptr;
   f.route_above = 0;
   f.seq_len = 0;

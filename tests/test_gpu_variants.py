@@ -95,3 +95,45 @@ def test_prefill_config_first_routed(pkg):
     g2 = run_ex(pkg, W.cuda(), hid.h, wl.tau, route_above=True, seq_len=512)
     assert np.array_equal(g2["route_mask"], planted.astype(np.uint8))
     assert np.array_equal(g2["first"], O.first_routed(planted.astype(np.uint8), 512))
+
+
+@pytest.mark.parametrize("n,d,dh", [(50, 128, 96), (700, 896, 256), (33, 36, 300)])
+def test_learned_router_score(pkg, n, d, dh):
+    V = 3000
+    W = S.make_W(d, V, seed=3, std=0.1)
+    hid = S.make_h(n, d, seed=5)
+    g = torch.Generator().manual_seed(dh)
+    W1 = (torch.randn(dh, d, generator=g) / d ** 0.5).to(torch.bfloat16)
+    b1 = torch.randn(dh, generator=g) * 0.1
+    w2 = torch.randn(dh, generator=g) * 0.5
+    b2 = 0.2
+    ref_score = O.mlp_router_score(S.bf16_bits(hid.h), S.bf16_bits(W1), b1.numpy(), w2.numpy(), b2)
+    base = O.route_oracle(S.bf16_bits(hid.h), S.bf16_bits(W), 0.5)
+    tau = float(np.median(ref_score))
+    want = O.route_decision(ref_score, tau)
+
+    r = pkg.Router(W.cuda(), max_n=n)
+    with pytest.raises(pkg.TlrError):                      # no router attached yet
+        r.route(hid.h.cuda(), tau, score_source=pkg.TLR_SCORE_MLP)
+    r.set_router_mlp(W1.cuda(), b1.cuda(), w2.cuda(), b2)
+    scores = torch.full((n,), float("nan"), device="cuda")
+    r.route(hid.h.cuda(), tau, score_source=pkg.TLR_SCORE_MLP, mlp_score=scores)
+    torch.cuda.synchronize()
+    assert pkg.tlr_last_device_status(r.ctx) == 0
+    got = scores.cpu().numpy()
+    assert np.max(np.abs(got - ref_score)) <= 1e-3
+    mask = r.route_mask[:n].cpu().numpy()
+    near = np.abs(ref_score - tau) <= 1e-3
+    assert np.array_equal(mask[~near], want[0][~near])
+    assert np.array_equal(mask == 1, got < np.float32(tau))          # decided on the learned score
+    c = int(r.routed_count.item())
+    assert c == int(mask.sum()) and np.array_equal(r.routed_idx[:c].cpu().numpy(), np.flatnonzero(mask))
+    assert 0 < c < n
+    # token / conf / entropy are still the LM head's
+    assert np.array_equal(r.token[:n].cpu().numpy()[base.top2_gap >= 1e-3], base.token[base.top2_gap >= 1e-3])
+    assert np.max(np.abs(r.conf[:n].cpu().numpy() - base.conf)) <= 1e-3
+    # the score alone, decision still on the confidence
+    r.route(hid.h.cuda(), 0.5, mlp_score=scores)
+    torch.cuda.synchronize()
+    assert np.array_equal(r.route_mask[:n].cpu().numpy(), base.route_mask)
+    r.close()

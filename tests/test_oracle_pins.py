@@ -304,3 +304,26 @@ def test_first_routed_position_per_sequence():
         assert f == (seg.min() - 12 * b if seg.size else 12)
     with pytest.raises(ValueError):
         O.first_routed(mask, 5)
+
+
+# ---------------------------------------------------------------- learned router score (shape assumed, not the paper's)
+def test_mlp_router_score_closed_forms_and_library():
+    h = bits_of([[1, 2], [-1, 0], [0, 0]])
+    W1 = bits_of([[1, 0], [0, 1], [-1, -1]])            # hidden = relu([h0, h1, -h0-h1] + b1)
+    b1 = np.array([0.0, 0.5, 0.0], np.float32)
+    w2 = np.array([1.0, -2.0, 3.0], np.float32)
+    s = O.mlp_router_score(h, W1, b1, w2, 0.25)
+    # row 0: hidden (1, 2.5, 0) -> 1 - 5 + 0 + .25 = -3.75; row 1: hidden (0, .5, 1) -> -1 + 3 + .25 = 2.25;
+    # row 2: hidden (0, .5, 0) -> -1 + .25 = -0.75                                  (worked by hand)
+    expect = [1 / (1 + math.exp(3.75)), 1 / (1 + math.exp(-2.25)), 1 / (1 + math.exp(0.75))]
+    np.testing.assert_allclose(s, expect, rtol=1e-14)
+    # zero output weights: sigmoid(b2) for every row
+    np.testing.assert_allclose(O.mlp_router_score(h, W1, b1, np.zeros(3, np.float32), 0.0), 0.5)
+    # independent library evaluation
+    g = torch.Generator().manual_seed(2)
+    hh = torch.randn(7, 24, generator=g).to(torch.bfloat16)
+    WW = torch.randn(40, 24, generator=g).to(torch.bfloat16)
+    bb = torch.randn(40, generator=g); ww = torch.randn(40, generator=g)
+    lib = torch.sigmoid(torch.relu(hh.double() @ WW.double().t() + bb.double()) @ ww.double() - 0.3)
+    got = O.mlp_router_score(S.bf16_bits(hh), S.bf16_bits(WW), bb.numpy(), ww.numpy(), -0.3)
+    np.testing.assert_allclose(got, lib.numpy(), rtol=1e-7)    # -0.3 is rounded to fp32 inside the oracle
