@@ -201,6 +201,16 @@ tlr_status tlr_last_device_status(tlr_ctx* ctx, uint32_t* out_host);
  * if the shape cannot run on the requested path. */
 tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path);
 
+/*
+ * tlr_debug_inject -- test hook for the kernels' failure handling.  Every barrier wait inside
+ * the projection kernel is bounded; when one runs out the kernel raises TLR_DEV_WAIT_TIMEOUT,
+ * lets its copies in flight land, frees its tensor memory and returns, and the context stays
+ * usable.  kind = 1 makes the next calls' W producer issue no copies, so the consumer's wait
+ * runs out (nothing faults, traps or spins forever); wait_limit_ms shortens the limit of every
+ * wait (0 = default, 2 s).  kind = 0 restores normal operation.  Tensor-core path only.
+ */
+tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms);
+
 /* tlr_plan_query -- the launch plan a call with n rows would use.  No device work. */
 tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out);
 

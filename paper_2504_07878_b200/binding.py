@@ -57,6 +57,8 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_route_ex.argtypes = [P, P, c_int32, c_float, POINTER(TlrRouteOptions), P, P, P, P, P, P, P]
     lib.tlr_route_ex.restype = c_int32
+    lib.tlr_debug_inject.argtypes = [P, c_int32, c_uint32]
+    lib.tlr_debug_inject.restype = c_int32
     lib.tlr_set_router_mlp.argtypes = [P, c_int32, P, P, P, c_float]
     lib.tlr_set_router_mlp.restype = c_int32
     lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
@@ -161,6 +163,11 @@ def tlr_last_device_status(ctx) -> int:
     out = c_uint32(0)
     _check(load_library().tlr_last_device_status(ctx, byref(out)), "tlr_last_device_status")
     return out.value
+
+
+def tlr_debug_inject(ctx, kind: int, wait_limit_ms: int = 0):
+    """Test hook: kind=1 drops the W copies of the next calls so a bounded wait runs out; kind=0 restores."""
+    _check(load_library().tlr_debug_inject(ctx, kind, wait_limit_ms), "tlr_debug_inject")
 
 
 def tlr_set_path(ctx, path: int):

@@ -84,6 +84,10 @@ struct tlr_ctx {
   float* mlp_scores = nullptr;     // [max_n][hidden blocks] partial sums of the output layer
   int mlp_blocks_cap = 0;
 
+  // test hook (tlr_debug_inject)
+  int debug_kind = 0;
+  unsigned long long debug_wait_ns = 0;
+
   bool timing = false;
   std::vector<cudaEvent_t> events;   // pairs, created lazily
   int timed = 0;
@@ -267,6 +271,13 @@ tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf1
   return TLR_OK;
 }
 
+tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms) {
+  if (ctx == nullptr || (kind != 0 && kind != 1)) return TLR_ERR_ARG;
+  ctx->debug_kind = kind;
+  ctx->debug_wait_ns = static_cast<unsigned long long>(wait_limit_ms) * 1000000ull;
+  return TLR_OK;
+}
+
 tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path) {
   if (ctx == nullptr) return TLR_ERR_ARG;
   if (path != TLR_PATH_AUTO && path != TLR_PATH_SIMT && path != TLR_PATH_TC) return TLR_ERR_ARG;
@@ -343,6 +354,8 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
       p.a_rows = cfg.a_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;
+      p.wait_limit_ns = ctx->debug_wait_ns;
+      p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
       p.partials = ctx->partials;
       p.status = ctx->status;
       e = tlr::launch_tc_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);

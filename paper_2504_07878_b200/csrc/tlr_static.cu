@@ -151,6 +151,8 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
       p.a_rows = cfg.a_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;
+      p.wait_limit_ns = 0;
+      p.debug_drop_w_copies = 0;
       p.partials = partials;
       p.status = status;
       if (tlr::launch_tc_projection(map_h, map_w128, map_w64, map_w16, p, cfg, units < workers_max ? units : workers_max,

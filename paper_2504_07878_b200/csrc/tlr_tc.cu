@@ -140,14 +140,14 @@ __device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
 
 // Bounded wait.  Returns false when the limit expired or another role already gave up.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* status) {
+                                          uint32_t* status, unsigned long long limit_ns) {
   if (mbar_try_wait(bar, parity)) return true;
   const unsigned long long t0 = global_ns();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 63u) == 0u) {
       if (*abort_flag) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         *abort_flag = 1;
         atomicOr(status, TLR_DEV_WAIT_TIMEOUT);
         return false;
@@ -381,6 +381,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   const int k_slabs = (p.d + kBlockK - 1) / kBlockK;
   const int units = p.chunks * p.row_units;
   const int T = p.tiles_per_unit;
+  const unsigned long long wait_ns = p.wait_limit_ns != 0 ? p.wait_limit_ns : kWaitLimitNs;
 
   if (warp == 0) {
     // ------------------------------------------------------------------ W producer
@@ -397,10 +398,11 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
             if (slab >= SB) {     // the stage is free once slab - SB has been consumed
               const int j = slab - SB;
-              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status)) { ok = false; break; }
+              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status, wait_ns)) { ok = false; break; }
             }
             const uint32_t dst = b_ring + stage * b_stage_bytes;
             const uint32_t bar = (kCta == 2) ? map_to_cta(b_full(stage), 0) : b_full(stage);
+            if (p.debug_drop_w_copies) continue;   // test hook: the copies are "lost", the consumer's wait runs out
             if (leader) mbar_expect_tx(b_full(stage), tl.rows * kRowBytes);   // both CTAs' bytes
             int r = 0;
             for (; my_rows - r >= 128; r += 128)
@@ -428,7 +430,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
             if (slab >= SA) {
               const int j = slab - SA;
-              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status)) { ok = false; break; }
+              if (!mbar_wait(released(j & (kRelease - 1)), (j / kRelease) & 1, abort_flag, p.status, wait_ns)) { ok = false; break; }
             }
             const uint32_t dst = a_ring + stage * a_stage_bytes;
             const uint32_t bar = (kCta == 2) ? map_to_cta(a_full(stage), 0) : a_full(stage);
@@ -466,14 +468,14 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           const Tile tl = tile_of<kCta>(p, unit, t, 0);
           if (tl.rows == 0) continue;
           const uint32_t idesc = instr_desc(kBlockM * kCta, tl.rows);
-          ok = __all_sync(0xffffffffu, mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status));
+          ok = __all_sync(0xffffffffu, mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status, wait_ns));
           if (!ok) break;
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + acc * kBlockN;
           for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
             if (!__all_sync(0xffffffffu, ra && rb)) {
-              const bool got = mbar_wait(a_full(sa), pa, abort_flag, p.status) &&
-                               mbar_wait(b_full(sb), pb, abort_flag, p.status);
+              const bool got = mbar_wait(a_full(sa), pa, abort_flag, p.status, wait_ns) &&
+                               mbar_wait(b_full(sb), pb, abort_flag, p.status, wait_ns);
               ok = __all_sync(0xffffffffu, got);
               if (!ok) break;
             }
@@ -523,7 +525,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
         if (tl.rows == 0) continue;
         const int v0 = tl.v0;
         const int cols = min(tl.rows, p.V - v0);   // valid columns of this tile
-        if (!mbar_wait(acc_full(acc), acc_phase, abort_flag, p.status)) { ok = false; break; }
+        if (!mbar_wait(acc_full(acc), acc_phase, abort_flag, p.status, wait_ns)) { ok = false; break; }
         tc_fence_after();
         if (warp_has_rows) {
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kBlockN;

@@ -29,6 +29,8 @@ struct TcParams {
   int n, d, V;
   int row_units, chunks, granules, tiles_per_unit;
   int a_rows, a_stages, b_stages;
+  unsigned long long wait_limit_ns;   // 0 = the default limit of every barrier wait
+  int debug_drop_w_copies;            // test hook: the W producer issues no copies
   Partial* partials;  // [n][chunks]
   uint32_t* status;
 };

@@ -204,3 +204,22 @@ def test_argument_errors(pkg):
                       router.route_mask, router.routed_idx, router.routed_count)
     assert e.value.code == 2
     router.close()
+
+
+@pytest.mark.parametrize("path", PATHS)
+def test_degenerate_vocabulary_and_tiny_shapes(pkg, path):
+    # V = 1: the only token has probability 1, entropy 0, and is never "below" any tau <= 1
+    W = S.make_W(8, 1, seed=1, std=0.5)
+    hid = S.make_h(5, 8, seed=1)
+    gpu = run_gpu(pkg, W.cuda(), hid.h, 1.0, path=path)
+    assert gpu["token"].tolist() == [0] * 5 and np.all(np.abs(gpu["conf"] - 1.0) < 1e-6) and np.all(gpu["entropy"] < 1e-6)
+    assert gpu["routed_count"] == 0
+    # V = 17 (one row past a 16-row granule), d = 16; and d = 8 with n past one row unit
+    for n, d, V in ((5, 16, 17), (200, 8, 33), (129, 8, 16)):
+        W = S.make_W(d, V, seed=V, std=0.7)
+        hid = S.make_h(n, d, seed=n)
+        ref = O.route_oracle(S.bf16_bits(hid.h), S.bf16_bits(W), 0.3)
+        gpu = run_gpu(pkg, W.cuda(), hid.h, 0.3, path=path)
+        assert gpu["status"] == 0
+        check_self_consistency(gpu, 0.3, V)
+        check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), O.bf16_bits_to_f64(S.bf16_bits(W)))
