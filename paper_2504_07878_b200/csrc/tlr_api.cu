@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdlib>
 #include <new>
 #include <vector>
 
@@ -42,6 +43,17 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
   plan->granule_rows = g;
   plan->granules = granules;
   plan->tiles_per_unit = best_tiles;
+  // How a unit's chunk is cut into tiles.  A tile costs a pass over all of h whatever its width,
+  // so where the tensor pipe matters (pairs of CTAs, n > 128) the chunk is cut into full 256-row
+  // tiles plus one remainder tile.  With one CTA per worker the path is HBM-bound and a narrow
+  // remainder tile only lowers the bytes in flight, so the tiles are of equal size there.
+  plan->full_tiles_first = 0;
+  if (cta == 2 && getenv("TLR_TC_EVEN_TILES") == nullptr) {   // (the variable is a tuning switch)
+    const long long gmax = (granules + best - 1) / best;
+    const long long full = 256 / g;
+    plan->full_tiles_first = 1;
+    plan->tiles_per_unit = static_cast<int>((gmax + full - 1) / full);
+  }
 }
 
 }  // namespace tlr
@@ -351,6 +363,7 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
       p.chunks = tp.chunks;
       p.granules = tp.granules;
       p.tiles_per_unit = tp.tiles_per_unit;
+      p.full_tiles_first = tp.full_tiles_first;
       p.a_rows = cfg.a_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;

@@ -301,8 +301,17 @@ __device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int 
   const int g0 = static_cast<int>((static_cast<long long>(p.granules) * r.chunk) / p.chunks);
   const int g1 = static_cast<int>((static_cast<long long>(p.granules) * (r.chunk + 1)) / p.chunks);
   const int G = g1 - g0;
-  const int ga = (G * t) / p.tiles_per_unit;
-  const int gb = (G * (t + 1)) / p.tiles_per_unit;
+  int ga, gb;
+  if (p.full_tiles_first) {
+    // as many full 256-row tiles as fit, then one remainder tile: a tile costs a pass over all
+    // of h whatever its width, so the fewest, widest tiles are the cheapest
+    const int full = kBlockN / (16 * kCta);
+    ga = min(G, full * t);
+    gb = min(G, full * (t + 1));
+  } else {
+    ga = (G * t) / p.tiles_per_unit;
+    gb = (G * (t + 1)) / p.tiles_per_unit;
+  }
   r.v0 = (g0 + ga) * (16 * kCta);
   r.rows = (gb - ga) * (16 * kCta);
   return r;

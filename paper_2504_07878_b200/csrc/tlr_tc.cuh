@@ -23,11 +23,12 @@ struct TcPlan {
   int granule_rows;    // 16 * cta
   int granules;        // ceil(V / granule_rows)
   int tiles_per_unit;  // every unit is walked in this many tiles (<= 256 rows each)
+  int full_tiles_first;  // 1: full 256-row tiles, then one remainder tile; 0: tiles of equal size
 };
 
 struct TcParams {
   int n, d, V;
-  int row_units, chunks, granules, tiles_per_unit;
+  int row_units, chunks, granules, tiles_per_unit, full_tiles_first;
   int a_rows, a_stages, b_stages;
   unsigned long long wait_limit_ns;   // 0 = the default limit of every barrier wait
   int debug_drop_w_copies;            // test hook: the W producer issues no copies
