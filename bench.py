@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_source": "paper_2504_07878_b200/csrc/tlr_tc.cu",
-    "sha256": "2f5ad762fe08c2e7344f78b141a4651eae56680604f18d26bb3464642656c7bb",
-    "bytes_per_launch": {"decode256": 276.68e6, "decode16": 276.32e6, "sweep512": 533.06e6},
+    "sha256": "2f31911b5719c35e32081a62015cd7ffec308f405482eb171bdf48bd4b9c09f0",
+    "bytes_per_launch": {"decode256": 276.68e6, "decode16": 275.94e6, "sweep512": 531.71e6},
 }
 
 
