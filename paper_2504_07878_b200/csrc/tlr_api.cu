@@ -19,7 +19,11 @@ constexpr int kMaxTimedLaunches = 4096;
 // number of chunks minimises (waves of units) x (rows of the largest chunk + a fixed cost
 // per tile), so that workers finish together.
 void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
-  const int g = 16 * cta;
+  int g = 16 * cta;
+  if (const char* env = getenv("TLR_TC_GRANULE")) {   // tuning switch
+    const int e = atoi(env);
+    if (e >= g && e <= 256 && e % g == 0 && 256 % e == 0) g = e;
+  }
   const int row_units = (n + 128 * cta - 1) / (128 * cta);
   const int granules = (V + g - 1) / g;
   int hi = granules < max_chunks ? granules : max_chunks;
@@ -283,6 +287,40 @@ tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf1
   return TLR_OK;
 }
 
+tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t* out, int32_t capacity,
+                                int32_t* count, tlr_plan* plan_out) {
+  if (n <= 0 || V <= 0 || sm_count < 2 || count == nullptr || capacity < 0 || (capacity > 0 && out == nullptr))
+    return TLR_ERR_ARG;
+  tlr::TcConfig cfg;
+  tlr::TcPlan tp;
+  tlr::tc_configure(n, &cfg);
+  const int workers_max = sm_count / cfg.cta;
+  tlr::tc_plan(n, V, cfg.cta, workers_max, tlr::kMaxChunks, &tp);
+  const int units = tp.chunks * tp.row_units;
+  const int workers = units < workers_max ? units : workers_max;
+  tlr::TcParams p = {};
+  p.n = n;
+  p.V = V;
+  p.row_units = tp.row_units;
+  p.chunks = tp.chunks;
+  p.granules = tp.granules;
+  p.tiles_per_unit = tp.tiles_per_unit;
+  p.full_tiles_first = tp.full_tiles_first;
+  p.granule_rows = tp.granule_rows;
+  *count = tlr::tc_enumerate_tiles(p, cfg.cta, workers, out, capacity);
+  if (plan_out != nullptr) {
+    plan_out->path = TLR_PATH_TC;
+    plan_out->grid = workers * cfg.cta;
+    plan_out->block = tlr::tc_threads();
+    plan_out->row_units = tp.row_units;
+    plan_out->vocab_chunks = tp.chunks;
+    plan_out->smem_bytes = cfg.smem_bytes;
+    plan_out->launches = 2;
+    plan_out->reserved = tp.granule_rows;
+  }
+  return TLR_OK;
+}
+
 tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms) {
   if (ctx == nullptr || (kind != 0 && kind != 1)) return TLR_ERR_ARG;
   ctx->debug_kind = kind;
@@ -364,6 +402,7 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
       p.granules = tp.granules;
       p.tiles_per_unit = tp.tiles_per_unit;
       p.full_tiles_first = tp.full_tiles_first;
+      p.granule_rows = tp.granule_rows;
       p.a_rows = cfg.a_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;

@@ -149,6 +149,7 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
       p.granules = tp.granules;
       p.tiles_per_unit = tp.tiles_per_unit;
       p.full_tiles_first = tp.full_tiles_first;
+      p.granule_rows = tp.granule_rows;
       p.a_rows = cfg.a_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;

@@ -11,7 +11,7 @@
 //             per 256 token rows.                                   (n > 128)
 //
 // Decomposition.  The vocabulary is cut into `chunks` contiguous ranges of granules
-// (16 * kCta rows); the token rows into units of 128 * kCta.  A work unit is
+// (a multiple of 16 * kCta rows); the token rows into units of 128 * kCta.  A work unit is
 // (chunk, row unit); units are numbered chunk-major so that workers running at the
 // same time share W through L2, and worker w takes units w, w + workers, ...  Inside
 // a unit the chunk is walked in `tiles_per_unit` tiles of at most 256 vocabulary rows
@@ -293,7 +293,7 @@ struct Tile {
 };
 
 template <int kCta>
-__device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int cta_rank) {
+__host__ __device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int cta_rank) {
   Tile r;
   r.chunk = unit / p.row_units;
   const int ru = unit - r.chunk * p.row_units;
@@ -305,15 +305,15 @@ __device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int 
   if (p.full_tiles_first) {
     // as many full 256-row tiles as fit, then one remainder tile: a tile costs a pass over all
     // of h whatever its width, so the fewest, widest tiles are the cheapest
-    const int full = kBlockN / (16 * kCta);
-    ga = min(G, full * t);
-    gb = min(G, full * (t + 1));
+    const int full = kBlockN / p.granule_rows;
+    ga = full * t < G ? full * t : G;
+    gb = full * (t + 1) < G ? full * (t + 1) : G;
   } else {
     ga = (G * t) / p.tiles_per_unit;
     gb = (G * (t + 1)) / p.tiles_per_unit;
   }
-  r.v0 = (g0 + ga) * (16 * kCta);
-  r.rows = (gb - ga) * (16 * kCta);
+  r.v0 = (g0 + ga) * p.granule_rows;
+  r.rows = (gb - ga) * p.granule_rows;
   return r;
 }
 
@@ -623,6 +623,31 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
 }
 
 int tc_threads() { return kThreads; }
+
+// Host enumeration of the schedule the kernel walks (the same tile_of the device code uses):
+// one record {worker, unit, row0, v0, rows} per non-empty tile of CTA rank 0, in walking order.
+int tc_enumerate_tiles(const TcParams& p, int cta, int workers, int* out, int capacity) {
+  int count = 0;
+  const int units = p.chunks * p.row_units;
+  for (int w = 0; w < workers; ++w) {
+    for (int unit = w; unit < units; unit += workers) {
+      for (int t = 0; t < p.tiles_per_unit; ++t) {
+        const Tile tl = cta == 2 ? tile_of<2>(p, unit, t, 0) : tile_of<1>(p, unit, t, 0);
+        if (tl.rows == 0) continue;
+        if (count < capacity) {
+          int* r = out + 5 * count;
+          r[0] = w;
+          r[1] = unit;
+          r[2] = tl.row0;
+          r[3] = tl.v0;
+          r[4] = tl.rows;
+        }
+        ++count;
+      }
+    }
+  }
+  return count;
+}
 
 // Ring depths and shared-memory size for a given n.  The h ring is short (L2 latency),
 // the W ring takes everything that is left (HBM latency).

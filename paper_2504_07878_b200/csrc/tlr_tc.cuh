@@ -20,7 +20,7 @@ struct TcConfig {
 struct TcPlan {
   int row_units;       // ceil(n / (128 * cta))
   int chunks;          // vocabulary chunks == partials per row
-  int granule_rows;    // 16 * cta
+  int granule_rows;    // a multiple of 16 * cta
   int granules;        // ceil(V / granule_rows)
   int tiles_per_unit;  // every unit is walked in this many tiles (<= 256 rows each)
   int full_tiles_first;  // 1: full 256-row tiles, then one remainder tile; 0: tiles of equal size
@@ -28,7 +28,7 @@ struct TcPlan {
 
 struct TcParams {
   int n, d, V;
-  int row_units, chunks, granules, tiles_per_unit, full_tiles_first;
+  int row_units, chunks, granules, tiles_per_unit, full_tiles_first, granule_rows;
   int a_rows, a_stages, b_stages;
   unsigned long long wait_limit_ns;   // 0 = the default limit of every barrier wait
   int debug_drop_w_copies;            // test hook: the W producer issues no copies
@@ -37,6 +37,7 @@ struct TcParams {
 };
 
 int tc_threads();
+int tc_enumerate_tiles(const TcParams& p, int cta, int workers, int* out, int capacity);
 void tc_configure(int n, TcConfig* c);
 void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan);
 cudaError_t tc_prepare();   // opt in to the kernels' dynamic shared memory size (once per device)
