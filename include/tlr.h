@@ -83,7 +83,8 @@ typedef struct {
  *   max_n       largest n any later call will pass (>= 1).  Sizes the workspace.
  *   out         receives the context.
  * The only call that allocates device memory: the per-row partial-result workspace,
- * a status word, and staging buffers for tlr_route_host.  Uses the current CUDA device.
+ * a status word, and staging buffers for tlr_route_host.  Uses the current CUDA device;
+ * every later call on the context must be made with that device current.
  * Errors: TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED (not an sm_100 device),
  * TLR_ERR_NOMEM, TLR_ERR_CUDA.  On error *out is NULL and nothing is leaked.
  */
@@ -178,7 +179,8 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
  * pointers may be NULL to skip that copy, except routed_count_host.  routed_idx_host
  * needs capacity n; only the first *routed_count_host entries are written.
  * Same errors as tlr_route, plus TLR_ERR_DEVICE_STATUS when a kernel raised
- * TLR_DEV_WAIT_TIMEOUT (outputs are then not to be trusted).
+ * TLR_DEV_WAIT_TIMEOUT (outputs are then not to be trusted).  The flag stays raised, and
+ * this call keeps returning that code, until tlr_last_device_status has read it.
  */
 tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau,
                           int32_t* token_host, float* conf_host, float* entropy_host,

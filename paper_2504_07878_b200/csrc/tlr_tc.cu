@@ -258,6 +258,32 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// Packed pairs of fp32 (one instruction works on both lanes) and the three-input maximum:
+// they halve the epilogue's instruction count per logit.
+__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
+  uint64_t r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
+  uint64_t d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+  uint64_t d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+  float d;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+  return d;
+}
+
 __device__ __forceinline__ float ex2_approx(float x) {
   float y;
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -549,9 +575,9 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
               for (int j = 0; j < 32; ++j)
                 if (j >= valid) z[j] = -1.0e30f;   // finite, so 0 * y stays 0 below
             }
-            float cm = z[0];
+            float cm = fmaxf(z[0], z[1]);
 #pragma unroll
-            for (int j = 1; j < 32; ++j) cm = fmaxf(cm, z[j]);
+            for (int j = 2; j < 32; j += 2) cm = max3(cm, z[j], z[j + 1]);
             if (cm > m) {
               if (m != -INFINITY) {
                 const float dl = (cm - m) * kLog2e;       // > 0
@@ -568,18 +594,20 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
               idx = v0 + c0 + first_j;
             }
             const float neg_ml = -m * kLog2e;
-            float ls0 = 0.f, ls1 = 0.f, lt0 = 0.f, lt1 = 0.f;
+            const uint64_t log2e2 = pack2(kLog2e, kLog2e), neg_ml2 = pack2(neg_ml, neg_ml);
+            uint64_t ls2 = pack2(0.f, 0.f), lt2 = pack2(0.f, 0.f);
 #pragma unroll
             for (int j = 0; j < 32; j += 2) {
-              const float y0 = fmaf(z[j], kLog2e, neg_ml);
-              const float y1 = fmaf(z[j + 1], kLog2e, neg_ml);
-              const float e0 = ex2_approx(y0);
-              const float e1 = ex2_approx(y1);
-              ls0 += e0;
-              ls1 += e1;
-              lt0 = fmaf(e0, y0, lt0);
-              lt1 = fmaf(e1, y1, lt1);
+              const uint64_t y2 = fma2(pack2(z[j], z[j + 1]), log2e2, neg_ml2);   // (z - m) * log2(e)
+              float y0, y1;
+              unpack2(y2, y0, y1);
+              const uint64_t e2 = pack2(ex2_approx(y0), ex2_approx(y1));
+              ls2 = add2(ls2, e2);
+              lt2 = fma2(e2, y2, lt2);
             }
+            float ls0, ls1, lt0, lt1;
+            unpack2(ls2, ls0, ls1);
+            unpack2(lt2, lt0, lt1);
             {
               const float a = (ls0 + ls1) - cS;
               const float b = S + a;
