@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_source": "paper_2504_07878_b200/csrc/tlr_tc.cu",
-    "sha256": "2f31911b5719c35e32081a62015cd7ffec308f405482eb171bdf48bd4b9c09f0",
-    "bytes_per_launch": {"decode256": 276.68e6, "decode16": 275.94e6, "sweep512": 531.71e6},
+    "sha256": "5569f0968e058aa14d3d6ee60a7be20f74028dc1137f5e0013cf6a91a85b2038",
+    "bytes_per_launch": {"decode256": 277.44e6, "decode16": 278.07e6, "sweep512": 531.56e6},
 }
 
 
