@@ -83,7 +83,7 @@ typedef struct {
  *   max_n       largest n any later call will pass (>= 1).  Sizes the workspace.
  *   out         receives the context.
  * The only call that allocates device memory: the per-row partial-result workspace,
- * a status word, and staging buffers for tlr_route_host.  Uses the current CUDA device;
+ * a status word, and staging buffers (device and pinned host) for tlr_route_host.  Uses the current CUDA device;
  * every later call on the context must be made with that device current.
  * Errors: TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED (not an sm_100 device),
  * TLR_ERR_NOMEM, TLR_ERR_CUDA.  On error *out is NULL and nothing is leaked.
@@ -174,8 +174,9 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
 
 /*
  * tlr_route_host -- the same step with HOST buffers: copies h to the device, runs
- * tlr_route, copies the six results back, and synchronises the stream before
- * returning.  Host buffers may be pageable or pinned (pinned is faster).  Output
+ * tlr_route, brings the six results back in one copy to a pinned buffer of the context,
+ * synchronises the stream and hands them out to the caller's buffers.  Host buffers may
+ * be pageable or pinned (a pinned h is faster).  Not reentrant on one context.  Output
  * pointers may be NULL to skip that copy, except routed_count_host.  routed_idx_host
  * needs capacity n; only the first *routed_count_host entries are written.
  * Same errors as tlr_route, plus TLR_ERR_DEVICE_STATUS when a kernel raised

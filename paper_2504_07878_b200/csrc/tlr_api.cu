@@ -3,6 +3,7 @@
 #include <cuda_runtime.h>
 
 #include <cstdlib>
+#include <cstring>
 #include <new>
 #include <vector>
 
@@ -83,13 +84,11 @@ struct tlr_ctx {
   uint32_t* status = nullptr;
 
   // staging for tlr_route_host
+  // One device block holds the six outputs of a call back to back, so that one copy brings
+  // them all to a pinned host mirror: token[n] conf[n] entropy[n] routed_idx[n] count mask[n].
   void* h_stage = nullptr;
-  int32_t* token_stage = nullptr;
-  float* conf_stage = nullptr;
-  float* entropy_stage = nullptr;
-  uint8_t* mask_stage = nullptr;
-  int32_t* idx_stage = nullptr;
-  int32_t* count_stage = nullptr;
+  unsigned char* out_stage = nullptr;    // device, 17 * max_n + 8 bytes
+  unsigned char* out_pinned = nullptr;   // pinned host mirror of the same size, + 4 bytes for the status word
 
   // learned router (tlr_set_router_mlp)
   int mlp_hidden = 0;
@@ -161,12 +160,8 @@ void free_all(tlr_ctx* c) {
   cudaFree(c->ticket);
   cudaFree(c->status);
   cudaFree(c->h_stage);
-  cudaFree(c->token_stage);
-  cudaFree(c->conf_stage);
-  cudaFree(c->entropy_stage);
-  cudaFree(c->mask_stage);
-  cudaFree(c->idx_stage);
-  cudaFree(c->count_stage);
+  cudaFree(c->out_stage);
+  cudaFreeHost(c->out_pinned);
   cudaFree(c->mlp_scores);
   for (cudaEvent_t e : c->events) cudaEventDestroy(e);
   delete c;
@@ -218,12 +213,8 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
   ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->token_stage, np * 4) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->conf_stage, np * 4) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->entropy_stage, np * 4) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->mask_stage, np) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->idx_stage, np * 4) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->count_stage, 4) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
+  ok = ok && cudaMallocHost(&c->out_pinned, np * 17 + 8 + 4) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_all(c);
@@ -480,29 +471,32 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
   if (n > 0 &&
       cudaMemcpyAsync(ctx->h_stage, h_bf16_host, nn * ctx->d * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess)
     return TLR_ERR_CUDA;
-  const tlr_status st = tlr_route(ctx, ctx->h_stage, n, tau, ctx->token_stage, ctx->conf_stage, ctx->entropy_stage,
-                                  ctx->mask_stage, ctx->idx_stage, ctx->count_stage, cuda_stream);
+  // layout of the output block for this n (all offsets are multiples of 4)
+  const size_t off_conf = 4 * nn, off_ent = 8 * nn, off_idx = 12 * nn, off_count = 16 * nn, off_mask = 16 * nn + 4;
+  const size_t out_bytes = 17 * nn + 4;
+  unsigned char* dev = ctx->out_stage;
+  const tlr_status st = tlr_route(ctx, ctx->h_stage, n, tau, reinterpret_cast<int32_t*>(dev),
+                                  reinterpret_cast<float*>(dev + off_conf), reinterpret_cast<float*>(dev + off_ent),
+                                  dev + off_mask, reinterpret_cast<int32_t*>(dev + off_idx),
+                                  reinterpret_cast<int32_t*>(dev + off_count), cuda_stream);
   if (st != TLR_OK) return st;
-  bool ok = true;
+  unsigned char* pin = ctx->out_pinned;
+  uint32_t* pin_status = reinterpret_cast<uint32_t*>(pin + static_cast<size_t>(ctx->max_n) * 17 + 8);
+  if (cudaMemcpyAsync(pin, dev, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(pin_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess)
+    return TLR_ERR_CUDA;
+  int32_t count = 0;
+  memcpy(&count, pin + off_count, 4);
+  *routed_count_host = count;
   if (n > 0) {
-    if (token_host) ok = ok && cudaMemcpyAsync(token_host, ctx->token_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    if (conf_host) ok = ok && cudaMemcpyAsync(conf_host, ctx->conf_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    if (entropy_host) ok = ok && cudaMemcpyAsync(entropy_host, ctx->entropy_stage, nn * 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-    if (route_mask_host) ok = ok && cudaMemcpyAsync(route_mask_host, ctx->mask_stage, nn, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    if (token_host) memcpy(token_host, pin, 4 * nn);
+    if (conf_host) memcpy(conf_host, pin + off_conf, 4 * nn);
+    if (entropy_host) memcpy(entropy_host, pin + off_ent, 4 * nn);
+    if (route_mask_host) memcpy(route_mask_host, pin + off_mask, nn);
+    if (routed_idx_host && count > 0) memcpy(routed_idx_host, pin + off_idx, 4 * static_cast<size_t>(count));
   }
-  uint32_t dev_status = 0;
-  ok = ok && cudaMemcpyAsync(routed_count_host, ctx->count_stage, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-  ok = ok && cudaMemcpyAsync(&dev_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
-  ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
-  if (!ok) return TLR_ERR_CUDA;
-  const int32_t count = *routed_count_host;
-  if (routed_idx_host != nullptr && count > 0) {
-    if (cudaMemcpyAsync(routed_idx_host, ctx->idx_stage, static_cast<size_t>(count) * 4, cudaMemcpyDeviceToHost,
-                        stream) != cudaSuccess ||
-        cudaStreamSynchronize(stream) != cudaSuccess)
-      return TLR_ERR_CUDA;
-  }
-  if (dev_status & TLR_DEV_WAIT_TIMEOUT) return TLR_ERR_DEVICE_STATUS;
+  if (*pin_status & TLR_DEV_WAIT_TIMEOUT) return TLR_ERR_DEVICE_STATUS;
   return TLR_OK;
 }
 
