@@ -1,7 +1,7 @@
 // Merge of the per-chunk partial results, the scores, the route decision and the
 // ordered stream compaction of routed rows -- one launch.
 //
-// Per row (one warp): lanes stride the row's partials; a shuffle butterfly finds the
+// Per row (a group of lanes, a whole warp for large n): lanes stride the row's partials; a shuffle butterfly finds the
 // global maximum and its lowest index, each lane rescales its own partials to that
 // maximum once, and a second butterfly adds the sums.  Lane 0 writes token,
 // conf = 1/s, entropy = ln s - t/s and the route flag conf < tau (Sec. 3.1 of the
