@@ -17,15 +17,22 @@
 // a unit the chunk is walked in `tiles_per_unit` tiles of at most 256 vocabulary rows
 // (the MMA's N), each a K-loop over d in slabs of 64 elements.
 //
-// Roles (warp-specialised, 224 threads per CTA):
-//   warp 0   W producer: TMA loads of W slabs into a deep ring (W comes from HBM)
+// Roles (warp-specialised, 352 threads per CTA):
+//   warp 0   W producer: TMA loads of W slabs into a deep ring (W comes from HBM).  W never
+//            depends on the previous kernel in the stream, so this warp does not wait for it:
+//            under programmatic dependent launch the ring fills while that kernel finishes.
 //   warp 6   h producer: TMA loads of h slabs into a short ring (h comes from L2)
 //   warp 1   MMA issuer (leader CTA only): tcgen05.mma x4 per slab into one of two
 //            256-column TMEM accumulators; also owns TMEM alloc/free
-//   warps 2-5 epilogue: each owns 32 TMEM lanes (rows); reads the finished accumulator
-//            32 columns at a time and folds it into per-row (m, idx, S, T) registers
-//            while the next tile's MMAs run into the other accumulator.
-// At the end of a unit every row's summary is written as one 16-byte partial.
+//   warps 2-5 and 7-10  epilogue, two warps per TMEM lane quadrant (32 rows): the first
+//            group folds the lower half of a finished accumulator's columns, the second
+//            group the upper half, 32 columns at a time, into per-row (m, idx, S, T)
+//            registers while the next tile's MMAs run into the other accumulator.  Two
+//            warps per scheduler hide each other's tensor-memory load and exp latency, and
+//            the time between a worker's last MMA and its last partial -- which nothing
+//            overlaps -- halves.
+// At the end of a unit the second group hands its summary to the first through shared memory
+// and every row's summary is written as one 16-byte partial.
 //
 // How much of W a CTA keeps in flight decides its streaming rate (latency-bound
 // otherwise), so h slabs get their own small ring and, when n is small, a slab of only
@@ -43,6 +50,7 @@
 
 #include "tlr_common.cuh"
 #include "tlr_tc.cuh"
+#include "tlr_tc_ptx.cuh"
 
 namespace tlr {
 
@@ -54,260 +62,16 @@ constexpr int kBlockK = 64;                  // bf16 per slab row = 128 B = one 
 constexpr int kUmmaK = 16;
 constexpr int kRowBytes = kBlockK * 2;       // 128
 constexpr int kTmemCols = 512;
-constexpr int kEpiWarps = 4;
-constexpr int kThreads = 32 * 7;
+constexpr int kEpiWarps = 8;                 // two groups of four (one warp per TMEM lane quadrant each)
+constexpr int kThreads = 32 * 11;
 constexpr int kMaxAStages = 8;
 constexpr int kMaxBStages = 12;
 constexpr int kRelease = 16;                 // >= every ring depth (see the barrier notes in the kernel)
 constexpr int kBarrierBytes = 512;
+constexpr int kScratchBytes = kBlockM * 16;  // one Partial per row: hand-over between the epilogue groups
 constexpr int kSmemLimit = 232448;           // 227 KiB opt-in maximum per CTA
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
-constexpr unsigned long long kDrainNs = 200000ull;          // 200 us: far beyond any copy's flight time
 
-__device__ __forceinline__ uint32_t smem_u32(const void* p) {
-  return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
-  return t;
-}
-
-__device__ __forceinline__ uint32_t cluster_ctarank() {
-  uint32_t r;
-  asm volatile("mov.u32 %0, %cluster_ctarank;" : "=r"(r));
-  return r;
-}
-// Address of the same shared-memory offset in CTA `rank` of this cluster.
-__device__ __forceinline__ uint32_t map_to_cta(uint32_t addr, uint32_t rank) {
-  uint32_t r;
-  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(addr), "r"(rank));
-  return r;
-}
-// True in exactly one lane of a converged warp.
-__device__ __forceinline__ bool elect_one() {
-  uint32_t pred;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "elect.sync _|p, 0xffffffff;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(pred));
-  return pred != 0;
-}
-__device__ __forceinline__ void cluster_sync_all() {
-  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
-  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-// Arrive on a barrier given by a shared::cluster address (own CTA or the peer).
-__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar_cluster_addr) {
-  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_cluster_addr) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Non-blocking poll of the same condition.
-__device__ __forceinline__ bool mbar_test_wait(uint32_t bar, uint32_t parity) {
-  uint32_t ok;
-  asm volatile(
-      "{\n\t.reg .pred p;\n\t"
-      "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-      "selp.u32 %0, 1, 0, p;\n\t}"
-      : "=r"(ok)
-      : "r"(bar), "r"(parity)
-      : "memory");
-  return ok != 0;
-}
-
-// Bounded wait.  Returns false when the limit expired or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag,
-                                          uint32_t* status, unsigned long long limit_ns) {
-  if (mbar_try_wait(bar, parity)) return true;
-  const unsigned long long t0 = global_ns();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if ((it & 63u) == 0u) {
-      if (*abort_flag) return false;
-      if (global_ns() - t0 > limit_ns) {
-        *abort_flag = 1;
-        atomicOr(status, TLR_DEV_WAIT_TIMEOUT);
-        return false;
-      }
-    }
-  }
-}
-
-// After giving up: let copies that are still in flight land before the CTA may exit.
-__device__ __forceinline__ void drain_delay() {
-  const unsigned long long t0 = global_ns();
-  while (global_ns() - t0 < kDrainNs) {}
-}
-
-// Tiled 2-D TMA load into this CTA's shared memory; completion bytes are signalled on
-// `bar` (a shared::cluster address).  With kCta == 2 the barrier may belong to the peer
-// CTA of the pair, which the cta_group::2 form permits.
-template <int kCta>
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y) {
-  if (kCta == 1) {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-  } else {
-    asm volatile(
-        "cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes "
-        "[%0], [%1, {%3, %4}], [%2];"
-        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(bar), "r"(x), "r"(y)
-        : "memory");
-  }
-}
-
-template <int kCta>
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t cols) {
-  if (kCta == 1)
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-  else
-    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(cols) : "memory");
-}
-template <int kCta>
-__device__ __forceinline__ void tmem_relinquish() {
-  if (kCta == 1)
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-  else
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
-}
-template <int kCta>
-__device__ __forceinline__ void tmem_dealloc(uint32_t addr, uint32_t cols) {
-  if (kCta == 1)
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-  else
-    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(addr), "r"(cols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate.  With kCta == 2 the
-// instruction runs on both SMs of the pair: each uses its own A rows and accumulator,
-// and B is the concatenation of the two CTAs' halves.
-template <int kCta>
-__device__ __forceinline__ void umma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
-                                          uint32_t accumulate) {
-  if (kCta == 1) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  } else {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
-        : "memory");
-  }
-}
-// Arrive on an mbarrier once every MMA issued so far by this thread has completed.  With
-// kCta == 2 the arrival is delivered to the barrier at the same offset in both CTAs.
-template <int kCta>
-__device__ __forceinline__ void umma_commit(uint32_t bar) {
-  if (kCta == 1) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-  } else {
-    const uint16_t mask = 3;
-    asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"(mask)
-        : "memory");
-  }
-}
-
-// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives row (lane base + i).
-__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float* v) {
-  uint32_t* r = reinterpret_cast<uint32_t*>(v);
-  asm volatile(
-      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-        "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-        "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-        "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-      : "r"(taddr)
-      : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Packed pairs of fp32 (one instruction works on both lanes) and the three-input maximum:
-// they halve the epilogue's instruction count per logit.
-__device__ __forceinline__ uint64_t pack2(float lo, float hi) {
-  uint64_t r;
-  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-  return r;
-}
-__device__ __forceinline__ void unpack2(uint64_t v, float& lo, float& hi) {
-  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
-}
-__device__ __forceinline__ uint64_t fma2(uint64_t a, uint64_t b, uint64_t c) {
-  uint64_t d;
-  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
-  return d;
-}
-__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
-  uint64_t d;
-  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-  return d;
-}
-__device__ __forceinline__ float max3(float a, float b, float c) {
-  float d;
-  asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
-  return d;
-}
-
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, laid out
-// by TMA with the 128-byte swizzle: 8-row groups 1024 bytes apart (stride offset 64 in
-// 16-byte units), leading offset unused (1), descriptor version 1, layout code 2.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-  uint64_t dsc = 0;
-  dsc |= static_cast<uint64_t>((saddr & 0x3ffffu) >> 4);
-  dsc |= static_cast<uint64_t>(1) << 16;
-  dsc |= static_cast<uint64_t>(1024 >> 4) << 32;
-  dsc |= static_cast<uint64_t>(1) << 46;
-  dsc |= static_cast<uint64_t>(2) << 61;
-  return dsc;
-}
-
-// Instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = m_rows, N = n_cols.
-__device__ __forceinline__ uint32_t instr_desc(int m_rows, int n_cols) {
-  return (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(n_cols >> 3) << 17) |
-         (static_cast<uint32_t>(m_rows >> 4) << 24);
-}
 
 // The static schedule, identical in every role: worker w walks units w, w + workers, ...;
 // each unit is `tiles_per_unit` tiles (possibly empty ones when the chunk is short).
@@ -372,11 +136,16 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   auto released = [&](int j) { return bar_base + 8u * (kMaxAStages + kMaxBStages + j); };
   auto acc_full = [&](int b) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + b); };
   auto acc_empty = [&](int b) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + 2 + b); };
-  constexpr int kNumBarriers = kMaxAStages + kMaxBStages + kRelease + 4;
+  // xch_full[q]: the second epilogue group's summary of quadrant q is in the scratch block;
+  // xch_empty[q]: the first group has read it.
+  auto xch_full = [&](int q) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + 4 + q); };
+  auto xch_empty = [&](int q) { return bar_base + 8u * (kMaxAStages + kMaxBStages + kRelease + 8 + q); };
+  constexpr int kNumBarriers = kMaxAStages + kMaxBStages + kRelease + 12;
   static_assert(kNumBarriers * 8 + 16 <= kBarrierBytes, "barrier block too small");
   unsigned char* gen_base = smem_raw + (base - smem_u32(smem_raw));
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(gen_base + (bar_base - base) + 8 * kNumBarriers);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  Partial* scratch = reinterpret_cast<Partial*>(gen_base + (bar_base - base) + kBarrierBytes);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
@@ -392,6 +161,10 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     for (int b = 0; b < 2; ++b) {
       mbar_init(acc_full(b), 1);
       mbar_init(acc_empty(b), kEpiWarps * kCta);
+    }
+    for (int q = 0; q < 4; ++q) {
+      mbar_init(xch_full(q), 1);
+      mbar_init(xch_empty(q), 1);
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -409,8 +182,9 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   // Programmatic dependent launch: everything above overlapped the tail of the previous
   // kernel in the stream; from here on its results (h, and the workspace the previous
   // merge kernel was still reading) are needed, so wait for it, then let the merge kernel
-  // that follows this one be scheduled early.
-  asm volatile("griddepcontrol.wait;" ::: "memory");
+  // that follows this one be scheduled early.  The W producer reads only W and the tensor
+  // maps, which no kernel writes, so it goes ahead.
+  if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
   const int k_slabs = (p.d + kBlockK - 1) / kBlockK;
@@ -540,13 +314,15 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
       }
     }
   } else {
-    // ------------------------------------------------------------------ epilogue (warps 2-5)
+    // ------------------------------------------------------------------ epilogue (warps 2-5, 7-10)
+    const int grp = warp >= 7 ? 1 : 0;       // 0: lower half of a tile's columns, 1: upper half
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
     const int row_in_cta = quad * 32 + lane;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
-    for (int unit = worker; unit < units && ok; unit += workers) {
+    uint32_t ord = 0;                        // ordinal of the unit among this worker's units
+    for (int unit = worker; unit < units && ok; unit += workers, ++ord) {
       const Tile first = tile_of<kCta>(p, unit, 0, cta_rank);
       const bool warp_has_rows = (first.row0 + quad * 32) < p.n;   // warp-uniform
       // Running summary of this thread's row over the unit.  S = sum 2^y and T = sum 2^y * y
@@ -560,11 +336,14 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
         if (tl.rows == 0) continue;
         const int v0 = tl.v0;
         const int cols = min(tl.rows, p.V - v0);   // valid columns of this tile
+        // this group's share of them: [0, half) or [half, cols), half a multiple of 32
+        const int half = min(cols, ((tl.rows / 2 + 31) / 32) * 32);
+        const int c_begin = grp ? half : 0, c_end = grp ? cols : half;
         if (!mbar_wait(acc_full(acc), acc_phase, abort_flag, p.status, wait_ns)) { ok = false; break; }
         tc_fence_after();
         if (warp_has_rows) {
           const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + acc * kBlockN;
-          for (int c0 = 0; c0 < cols; c0 += 32) {
+          for (int c0 = c_begin; c0 < c_end; c0 += 32) {
             float z[32];
             __syncwarp();                           // the load below is warp-collective
             tmem_ld32(taddr + c0, z);
@@ -630,13 +409,30 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
         }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
-      if (ok && first.row0 + row_in_cta < p.n) {
-        Partial out;
-        out.m = m;
-        out.idx = idx;
-        out.s = S;
-        out.t = Tq * kLn2;             // sum e^(z-m) (z-m), back in nats
-        p.partials[static_cast<size_t>(first.row0 + row_in_cta) * p.chunks + first.chunk] = out;
+      Partial out;
+      out.m = m;
+      out.idx = idx;
+      out.s = S;
+      out.t = Tq * kLn2;             // sum e^(z-m) (z-m), back in nats
+      // The second group hands its summary to the first through the scratch block (bounded
+      // waits on both sides: a warp that gave up never leaves its partner waiting forever).
+      if (grp == 1) {
+        if (ok && ord > 0) ok = mbar_wait(xch_empty(quad), (ord - 1) & 1u, abort_flag, p.status, wait_ns);
+        if (ok) {
+          scratch[row_in_cta] = out;
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xch_full(quad));
+        }
+      } else {
+        if (ok) ok = mbar_wait(xch_full(quad), ord & 1u, abort_flag, p.status, wait_ns);
+        if (ok) {
+          const Partial other = scratch[row_in_cta];
+          __syncwarp();
+          if (lane == 0) mbar_arrive(xch_empty(quad));
+          out = merge(out, other);
+          if (first.row0 + row_in_cta < p.n)
+            p.partials[static_cast<size_t>(first.row0 + row_in_cta) * p.chunks + first.chunk] = out;
+        }
       }
     }
   }
@@ -691,8 +487,8 @@ void tc_configure(int n, TcConfig* c) {
   const int b_stage = (kBlockN / cta) * kRowBytes;
   // h slabs come from L2 (about a microsecond away under load) and one is consumed per W
   // slab, so the h ring needs about half the depth of the W ring to keep up.
-  int sa = cta == 2 ? 5 : (a_rows <= 32 ? 6 : 4);
-  const int budget = kSmemLimit - 1024 - kBarrierBytes;
+  int sa = cta == 2 ? 4 : (a_rows <= 32 ? 6 : 4);
+  const int budget = kSmemLimit - 1024 - kBarrierBytes - kScratchBytes;
   int sb = (budget - sa * a_stage) / b_stage;
   if (sb > kMaxBStages) sb = kMaxBStages;
   // Tuning override: TLR_TC_RINGS="<h stages>,<W stages>" (ignored if it does not fit).
@@ -708,7 +504,7 @@ void tc_configure(int n, TcConfig* c) {
   c->a_rows = a_rows;
   c->a_stages = sa;
   c->b_stages = sb;
-  c->smem_bytes = 1024 + sa * a_stage + sb * b_stage + kBarrierBytes;
+  c->smem_bytes = 1024 + sa * a_stage + sb * b_stage + kBarrierBytes + kScratchBytes;
 }
 
 cudaError_t tc_prepare() {
