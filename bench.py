@@ -35,20 +35,22 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # captures summarised under profiles/.  Only valid for the kernel source they were taken on: the
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
-    "kernel_source": "paper_2504_07878_b200/csrc/tlr_tc.cu",
-    "sha256": "5569f0968e058aa14d3d6ee60a7be20f74028dc1137f5e0013cf6a91a85b2038",
-    "bytes_per_launch": {"decode256": 277.44e6, "decode16": 278.07e6, "sweep512": 531.56e6},
+    "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc.cu", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
+    "sha256": "f59fe13215d784aaaf9774ee28ea5f9e26f10523198f646fd29ff2e415568a33",
+    "bytes_per_launch": {"decode256": 276.86e6, "decode16": 276.26e6, "sweep512": 531.56e6},
 }
 
 
 def ncu_traffic(workload):
     import hashlib
-    path = os.path.join(ROOT, NCU_TRAFFIC["kernel_source"])
+    digest = hashlib.sha256()
     try:
-        with open(path, "rb") as f:
-            if hashlib.sha256(f.read()).hexdigest() != NCU_TRAFFIC["sha256"]:
-                return None
+        for rel in NCU_TRAFFIC["kernel_sources"]:
+            with open(os.path.join(ROOT, rel), "rb") as f:
+                digest.update(f.read())
     except OSError:
+        return None
+    if digest.hexdigest() != NCU_TRAFFIC["sha256"]:
         return None
     return NCU_TRAFFIC["bytes_per_launch"].get(workload)
 
