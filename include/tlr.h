@@ -173,6 +173,33 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
                         int32_t* routed_count_dev, void* cuda_stream);
 
 /*
+ * tlr_shard_summary / tlr_shard_finish -- the routing step with the vocabulary sharded over several
+ * GPUs (one process per GPU).  The paper decodes on one device; this is the data-parallel
+ * restatement for decode batches, where streaming W from HBM dominates the step (the LM-head
+ * contraction on the hidden state of Sec. 3.3, the decision of Sec. 3.1): GPU g holds the
+ * contiguous rows [v_offset, v_offset + V) of the full W, and its context is created on that block.
+ *
+ * tlr_shard_summary runs the projection over the shard and writes, for each of the n rows, one
+ * 16-byte summary {float m; int32 idx; float s; float t} into summary_dev[n] (device, 16-byte
+ * aligned, caller-owned): m = the largest logit in the shard, idx = the lowest GLOBAL vocabulary
+ * index attaining it (v_offset already added), s = sum exp(z - m), t = sum exp(z - m)(z - m) over
+ * the shard.  No decision is taken.  The caller then exchanges the summaries -- an all-gather of
+ * n x 16 bytes per GPU, NCCL in the Python helper -- into a block laid out [shards][n].
+ *
+ * tlr_shard_finish merges the `shards` summaries of every row (the same associative rule that merges
+ * the chunks of one GPU; ties go to the lower index), and produces the six outputs of tlr_route.
+ * Any context of the same max_n can run it; 1 <= shards <= 192.  Same ownership, stream and error
+ * rules as tlr_route; nothing is allocated.  The result differs from the one-GPU result only by
+ * fp32 summation order (conf and entropy agree to a few ulp; token, route_mask, routed_idx and
+ * routed_count are identical unless a row sits within rounding of a tie or of tau).
+ */
+tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, int32_t v_offset, void* summary_dev,
+                             void* cuda_stream);
+tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t shards, int32_t n, float tau,
+                            int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
+                            int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream);
+
+/*
  * tlr_route_host -- the same step with HOST buffers: copies h to the device, runs
  * tlr_route, brings the six results back in one copy to a pinned buffer of the context,
  * synchronises the stream and hands them out to the caller's buffers.  Host buffers may

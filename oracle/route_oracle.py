@@ -22,6 +22,9 @@ What it computes, per decoding position i (one row of ``h``):
   Variants of steps 5-6: one threshold per row, the opposite polarity (Sec. 2.2:
   defer when the score exceeds the threshold), and the first routed position of
   every sequence (Sec. 4.1: where the re-processing of a returned context stops).
+  Vocabulary-sharded form (several GPUs, each a contiguous range of W's rows):
+  shard_summary is what one range reports per row, merge_summaries combines the
+  ranges; together they must reproduce steps 2-4 (pinned against them).
 
 All arithmetic is fp64 on the exact values of the bf16 inputs.  The only
 library primitive used as a step is the dense matrix product of step 1.  Rows
@@ -161,6 +164,43 @@ def with_threshold(result: RouteResult, tau, route_above: bool = False) -> Route
     """The same per-row scores with steps 5-6 redone for another threshold or polarity."""
     mask, idx, count, tau32 = route_decision(result.conf, tau, route_above)
     return RouteResult(result.token, result.conf, result.entropy, mask, idx, count, result.top2_gap, tau32)
+
+
+def shard_summary(h_bits: np.ndarray, W_shard_bits: np.ndarray, v_offset: int):
+    """Per-row summary of a contiguous range of the vocabulary (rows v_offset.. of the full W).
+
+    What one GPU of a vocabulary-sharded step reports for a row with shard logits z:
+        m = max z,  idx = v_offset + lowest position attaining it,
+        s = sum exp(z - m),  t = sum exp(z - m) * (z - m).
+    Returned as four arrays (m, idx, s, t), fp64 / int64.
+    """
+    z = logits_fp64(bf16_bits_to_f64(h_bits), bf16_bits_to_f64(W_shard_bits))
+    m = z.max(axis=1)
+    idx = z.argmax(axis=1).astype(np.int64) + int(v_offset)
+    e = np.exp(z - m[:, None])
+    return m, idx, e.sum(axis=1), (e * (z - m[:, None])).sum(axis=1)
+
+
+def merge_summaries(parts):
+    """Combines per-row summaries of disjoint vocabulary ranges into token, conf, entropy.
+
+    With M the largest of the ranges' maxima: token = the lowest index among the ranges that
+    attain M; S = sum_g s_g exp(m_g - M); T = sum_g exp(m_g - M) (t_g + (m_g - M) s_g);
+    conf = 1/S and entropy = ln S - T/S.  (Both follow from p_v = exp(z_v - M)/S:
+    p_token = 1/S, and -sum p ln p = ln S - (1/S) sum exp(z_v - M)(z_v - M).)
+    """
+    ms = np.stack([p[0] for p in parts])            # [G, n]
+    idxs = np.stack([p[1] for p in parts])
+    M = ms.max(axis=0)
+    at_max = ms == M[None, :]
+    token = np.where(at_max, idxs, np.iinfo(np.int64).max).min(axis=0)
+    S = np.zeros_like(M)
+    T = np.zeros_like(M)
+    for m, _, s, t in parts:
+        w = np.exp(m - M)
+        S += s * w
+        T += w * (t + (m - M) * s)
+    return token.astype(np.int32), 1.0 / S, np.log(S) - T / S
 
 
 def mlp_router_score(h_bits: np.ndarray, W1_bits: np.ndarray, b1, w2, b2: float) -> np.ndarray:

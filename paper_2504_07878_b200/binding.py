@@ -64,6 +64,10 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_set_router_mlp.argtypes = [P, c_int32, P, P, P, c_float]
     lib.tlr_set_router_mlp.restype = c_int32
     lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_shard_summary.argtypes = [P, P, c_int32, c_int32, P, P]
+    lib.tlr_shard_summary.restype = c_int32
+    lib.tlr_shard_finish.argtypes = [P, P, c_int32, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_shard_finish.restype = c_int32
     lib.tlr_destroy.argtypes = [P]
     lib.tlr_status_string.argtypes = [c_int32]
     lib.tlr_status_string.restype = c_char_p
@@ -142,6 +146,20 @@ def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask,
     _check(load_library().tlr_route_host(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
                                          _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
                                          _stream_handle(stream)), "tlr_route_host")
+
+
+def tlr_shard_summary(ctx, h, n: int, v_offset: int, summary, stream=None):
+    """Vocabulary-sharded step, part 1: one 16-byte summary per row over this GPU's rows of W (global indices)."""
+    _check(load_library().tlr_shard_summary(ctx, _ptr(h), n, v_offset, _ptr(summary), _stream_handle(stream)),
+           "tlr_shard_summary")
+
+
+def tlr_shard_finish(ctx, summaries, shards: int, n: int, tau: float, token, conf, entropy, route_mask, routed_idx,
+                     routed_count, stream=None):
+    """Part 2: merge the gathered summaries [shards][n] and produce the six outputs of tlr_route."""
+    _check(load_library().tlr_shard_finish(ctx, _ptr(summaries), shards, n, tau, _ptr(token), _ptr(conf),
+                                           _ptr(entropy), _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
+                                           _stream_handle(stream)), "tlr_shard_finish")
 
 
 def tlr_route_static(d: int, V: int, W, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx,

@@ -167,6 +167,65 @@ void free_all(tlr_ctx* c) {
   delete c;
 }
 
+// Enqueues the projection kernel of a call with n > 0 rows: chunk partials into ctx->partials.
+tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const tlr_plan& plan, cudaStream_t stream) {
+  cudaEvent_t ev0 = nullptr, ev1 = nullptr;
+  if (ctx->timing && ctx->timed < tlr::kMaxTimedLaunches) {
+    const size_t need = 2 * static_cast<size_t>(ctx->timed + 1);
+    while (ctx->events.size() < need) {
+      cudaEvent_t e;
+      if (cudaEventCreate(&e) != cudaSuccess) return TLR_ERR_CUDA;
+      ctx->events.push_back(e);
+    }
+    ev0 = ctx->events[2 * ctx->timed];
+    ev1 = ctx->events[2 * ctx->timed + 1];
+    if (cudaEventRecord(ev0, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  }
+  cudaError_t e;
+  if (plan.path == TLR_PATH_TC) {
+    tlr::TcConfig cfg;
+    tlr::TcPlan tp;
+    tlr::tc_configure(n, &cfg);
+    tlr::tc_plan(n, ctx->V, cfg.cta, ctx->sm_count / cfg.cta, tlr::kMaxChunks, &tp);
+    CUtensorMap map_h;
+    if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
+    tlr::TcParams p;
+    p.n = n;
+    p.d = ctx->d;
+    p.V = ctx->V;
+    p.row_units = tp.row_units;
+    p.chunks = tp.chunks;
+    p.granules = tp.granules;
+    p.tiles_per_unit = tp.tiles_per_unit;
+    p.full_tiles_first = tp.full_tiles_first;
+    p.granule_rows = tp.granule_rows;
+    p.a_rows = cfg.a_rows;
+    p.a_stages = cfg.a_stages;
+    p.b_stages = cfg.b_stages;
+    p.wait_limit_ns = ctx->debug_wait_ns;
+    p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
+    p.partials = ctx->partials;
+    p.status = ctx->status;
+    e = tlr::launch_tc_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
+  } else {
+    tlr::SimtLaunch a;
+    a.W = ctx->W;
+    a.h = h_bf16_dev;
+    a.n = n;
+    a.d = ctx->d;
+    a.V = ctx->V;
+    a.chunks = plan.vocab_chunks;
+    a.partials = ctx->partials;
+    e = tlr::launch_simt_projection(a, stream);
+  }
+  if (e != cudaSuccess) return TLR_ERR_CUDA;
+  if (ev1 != nullptr) {
+    if (cudaEventRecord(ev1, stream) != cudaSuccess) return TLR_ERR_CUDA;
+    ctx->timed += 1;
+  }
+  return TLR_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -364,60 +423,8 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
   fill_plan(ctx, n, &plan);
 
   if (n > 0) {
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr;
-    if (ctx->timing && ctx->timed < tlr::kMaxTimedLaunches) {
-      const size_t need = 2 * static_cast<size_t>(ctx->timed + 1);
-      while (ctx->events.size() < need) {
-        cudaEvent_t e;
-        if (cudaEventCreate(&e) != cudaSuccess) return TLR_ERR_CUDA;
-        ctx->events.push_back(e);
-      }
-      ev0 = ctx->events[2 * ctx->timed];
-      ev1 = ctx->events[2 * ctx->timed + 1];
-      if (cudaEventRecord(ev0, stream) != cudaSuccess) return TLR_ERR_CUDA;
-    }
-    cudaError_t e;
-    if (plan.path == TLR_PATH_TC) {
-      tlr::TcConfig cfg;
-      tlr::TcPlan tp;
-      tlr::tc_configure(n, &cfg);
-      tlr::tc_plan(n, ctx->V, cfg.cta, ctx->sm_count / cfg.cta, tlr::kMaxChunks, &tp);
-      CUtensorMap map_h;
-      if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
-      tlr::TcParams p;
-      p.n = n;
-      p.d = ctx->d;
-      p.V = ctx->V;
-      p.row_units = tp.row_units;
-      p.chunks = tp.chunks;
-      p.granules = tp.granules;
-      p.tiles_per_unit = tp.tiles_per_unit;
-      p.full_tiles_first = tp.full_tiles_first;
-      p.granule_rows = tp.granule_rows;
-      p.a_rows = cfg.a_rows;
-      p.a_stages = cfg.a_stages;
-      p.b_stages = cfg.b_stages;
-      p.wait_limit_ns = ctx->debug_wait_ns;
-      p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
-      p.partials = ctx->partials;
-      p.status = ctx->status;
-      e = tlr::launch_tc_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
-    } else {
-      tlr::SimtLaunch a;
-      a.W = ctx->W;
-      a.h = h_bf16_dev;
-      a.n = n;
-      a.d = ctx->d;
-      a.V = ctx->V;
-      a.chunks = plan.vocab_chunks;
-      a.partials = ctx->partials;
-      e = tlr::launch_simt_projection(a, stream);
-    }
-    if (e != cudaSuccess) return TLR_ERR_CUDA;
-    if (ev1 != nullptr) {
-      if (cudaEventRecord(ev1, stream) != cudaSuccess) return TLR_ERR_CUDA;
-      ctx->timed += 1;
-    }
+    const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, plan, stream);
+    if (ps != TLR_OK) return ps;
   }
 
   if (want_mlp && n > 0) {
@@ -448,6 +455,59 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
   f.route_above = (opt != nullptr && opt->route_above != 0) ? 1 : 0;
   f.seq_len = opt != nullptr ? opt->seq_len : 0;
   f.first_routed = opt != nullptr ? opt->first_routed_dev : nullptr;
+  f.token = token_dev;
+  f.conf = conf_dev;
+  f.entropy = entropy_dev;
+  f.route_mask = route_mask_dev;
+  f.routed_idx = routed_idx_dev;
+  f.routed_count = routed_count_dev;
+  f.ticket = ctx->ticket;
+  f.status = ctx->status;
+  if (tlr::launch_finish(f, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, int32_t v_offset, void* summary_dev,
+                             void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || v_offset < 0) return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n == 0) return TLR_OK;
+  if (h_bf16_dev == nullptr || summary_dev == nullptr) return TLR_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(h_bf16_dev) & 15u) != 0 || (reinterpret_cast<uintptr_t>(summary_dev) & 15u) != 0)
+    return TLR_ERR_ALIGN;
+  if (static_cast<long long>(v_offset) + ctx->V + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  tlr_plan plan;
+  fill_plan(ctx, n, &plan);
+  const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, plan, stream);
+  if (ps != TLR_OK) return ps;
+  if (tlr::launch_shard_summary(ctx->partials, n, plan.vocab_chunks, v_offset, static_cast<Partial*>(summary_dev),
+                                stream) != cudaSuccess)
+    return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t shards, int32_t n, float tau,
+                            int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
+                            int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || routed_count_dev == nullptr || shards < 1 || shards > tlr::kMaxChunks)
+    return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n > 0) {
+    if (summaries_dev == nullptr || token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr ||
+        route_mask_dev == nullptr || routed_idx_dev == nullptr)
+      return TLR_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(summaries_dev) & 15u) != 0) return TLR_ERR_ALIGN;
+  }
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  if (tlr::launch_shard_gather(static_cast<const Partial*>(summaries_dev), shards, n, ctx->partials, stream) !=
+      cudaSuccess)
+    return TLR_ERR_CUDA;
+  tlr::FinishLaunch f = {};
+  f.partials = ctx->partials;
+  f.n = n;
+  f.chunks = shards;
+  f.tau = tau;
   f.token = token_dev;
   f.conf = conf_dev;
   f.entropy = entropy_dev;

@@ -112,6 +112,12 @@ struct FinishLaunch {
 };
 cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
 
+// Vocabulary-sharded decode (tlr_shard.cu): one summary per row from a shard's chunk partials,
+// and the gathered summaries [shards][n] laid out as partials [n][shards].
+cudaError_t launch_shard_summary(const Partial* partials, int n, int chunks, int v_offset, Partial* summary,
+                                 cudaStream_t stream);
+cudaError_t launch_shard_gather(const Partial* gathered, int shards, int n, Partial* partials, cudaStream_t stream);
+
 struct MlpLaunch {
   const void* h;        // bf16 [n][d]
   const void* W1;       // bf16 [d_hidden][d]

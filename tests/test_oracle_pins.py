@@ -327,3 +327,43 @@ def test_mlp_router_score_closed_forms_and_library():
     lib = torch.sigmoid(torch.relu(hh.double() @ WW.double().t() + bb.double()) @ ww.double() - 0.3)
     got = O.mlp_router_score(S.bf16_bits(hh), S.bf16_bits(WW), bb.numpy(), ww.numpy(), -0.3)
     np.testing.assert_allclose(got, lib.numpy(), rtol=1e-7)    # -0.3 is rounded to fp32 inside the oracle
+
+
+# ---------------------------------------------------------------- vocabulary-sharded form
+
+def test_shard_summaries_merge_to_the_plain_definition():
+    """Any contiguous partition of the vocabulary, summarised and merged, gives steps 2-4 of the
+    plain definition: token exactly (also when the maximum is tied across two ranges), conf and
+    entropy to rounding."""
+    rng = np.random.default_rng(5)
+    n, d, V = 9, 16, 211
+    h = S.bf16_bits(torch.from_numpy(rng.standard_normal((n, d)).astype(np.float32)).to(torch.bfloat16))
+    Wt = torch.from_numpy((0.3 * rng.standard_normal((V, d))).astype(np.float32)).to(torch.bfloat16)
+    Wt[20] = Wt[20] * 4.0                             # a long row, so that a hidden state along it peaks there
+    Wt[150] = Wt[20]                                  # ... and an exact copy of it in another range: a tie
+    hb = S.bf16_bits(Wt[20:21])                       # a row whose maximum is that tied pair
+    h = np.concatenate([h, hb], axis=0)
+    W = S.bf16_bits(Wt)
+    ref = O.route_oracle(h, W, 0.5)
+    for cuts in ([0, 211], [0, 100, 211], [0, 32, 64, 160, 211], [0, 1, 210, 211]):
+        parts = [O.shard_summary(h, W[a:b], a) for a, b in zip(cuts[:-1], cuts[1:])]
+        token, conf, ent = O.merge_summaries(parts)
+        assert np.array_equal(token, ref.token)
+        assert np.allclose(conf, ref.conf, rtol=1e-12, atol=0)
+        assert np.allclose(ent, ref.entropy, rtol=0, atol=1e-12)
+    assert ref.token[-1] == 20                        # the tie went to the lower index
+
+
+def test_shard_summary_hand_worked():
+    """Two ranges of a four-token vocabulary with integer logits: range A = {0, 2}, range B = {2, 1}."""
+    h = S.bf16_bits(torch.tensor([[1.0, 0.0]], dtype=torch.bfloat16))
+    W = S.bf16_bits(torch.tensor([[0.0, 5.0], [2.0, 1.0], [2.0, 7.0], [1.0, 3.0]], dtype=torch.bfloat16))
+    mA, iA, sA, tA = O.shard_summary(h, W[0:2], 0)
+    mB, iB, sB, tB = O.shard_summary(h, W[2:4], 2)
+    assert mA[0] == 2.0 and iA[0] == 1 and sA[0] == pytest.approx(1 + math.exp(-2)) and tA[0] == pytest.approx(-2 * math.exp(-2))
+    assert mB[0] == 2.0 and iB[0] == 2 and sB[0] == pytest.approx(1 + math.exp(-1)) and tB[0] == pytest.approx(-math.exp(-1))
+    token, conf, ent = O.merge_summaries([(mA, iA, sA, tA), (mB, iB, sB, tB)])
+    Ssum = 2 + math.exp(-2) + math.exp(-1)
+    assert token[0] == 1 and conf[0] == pytest.approx(1 / Ssum)
+    p = np.array([math.exp(-2), 1.0, 1.0, math.exp(-1)]) / Ssum
+    assert ent[0] == pytest.approx(float(-(p * np.log(p)).sum()))
