@@ -10,9 +10,15 @@
 // Compaction (ballot / popcount / prefix sum, ascending order):
 //   n <= 1024  a thread-block cluster of up to 8 blocks folds the rows (a group of L lanes
 //              per row, all rows at once); after a cluster barrier block 0 compacts the
-//              flags in one pass.  No ticket, no second launch, about two L2 round trips.
+//              flags.  No ticket, no second launch, about two L2 round trips.  The blocks
+//              have 512 threads where a lane group still owns at most 6 partials (else 1024):
+//              that size fits on an SM beside a CTA of the tensor-core projection kernel, so
+//              the blocks are resident and waiting before that kernel ends, and the next
+//              call's CTAs do not have to wait for the merge to leave their SMs.
 //   larger n   many blocks of 8 warps; the block that finishes last (fence + ticket
 //              counter, no spinning) compacts the flags of all rows.
+#include <cstdlib>
+
 #include "tlr_common.cuh"
 
 namespace tlr {
@@ -139,7 +145,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
   __shared__ int warp_count[kSmallThreads / 32];
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
-  const int group = (blockIdx.x * kSmallThreads + threadIdx.x) / L;
+  const int group = (blockIdx.x * blockDim.x + threadIdx.x) / L;
   const int gl = threadIdx.x & (L - 1);
   pdl_enter();
   __shared__ unsigned char flags[kSmallRows];
@@ -244,24 +250,29 @@ finish_small_kernel(const FinishLaunch a, const int L) {
   }
   if (blockIdx.x != 0) return;
   first_routed_init(a);
-  const int i = threadIdx.x;
-  int flag = 0;
-  if (i < a.n) flag = single_block ? static_cast<int>(flags[i]) : static_cast<int>(__ldcg(a.route_mask + i));
-  const unsigned int bal = __ballot_sync(0xffffffffu, flag != 0);
-  if (lane == 0) warp_count[warp] = __popc(bal);
-  __syncthreads();
-  int before = 0, total = 0;
-#pragma unroll
-  for (int w = 0; w < kSmallThreads / 32; ++w) {
-    const int c = warp_count[w];
-    before += (w < warp) ? c : 0;
-    total += c;
+  const int warps = blockDim.x >> 5;
+  int base_out = 0;
+  for (int base = 0; base < a.n; base += blockDim.x) {       // one pass when the block has a thread per row
+    const int i = base + threadIdx.x;
+    int flag = 0;
+    if (i < a.n) flag = single_block ? static_cast<int>(flags[i]) : static_cast<int>(__ldcg(a.route_mask + i));
+    const unsigned int bal = __ballot_sync(0xffffffffu, flag != 0);
+    if (lane == 0) warp_count[warp] = __popc(bal);
+    __syncthreads();
+    int before = 0, total = 0;
+    for (int w = 0; w < warps; ++w) {
+      const int c = warp_count[w];
+      before += (w < warp) ? c : 0;
+      total += c;
+    }
+    if (flag) {
+      a.routed_idx[base_out + before + __popc(bal & ((1u << lane) - 1u))] = i;
+      first_routed_note(a, i);
+    }
+    base_out += total;
+    __syncthreads();
   }
-  if (flag) {
-    a.routed_idx[before + __popc(bal & ((1u << lane) - 1u))] = i;
-    first_routed_note(a, i);
-  }
-  if (threadIdx.x == 0) *a.routed_count = total;
+  if (threadIdx.x == 0) *a.routed_count = base_out;
 }
 
 __global__ void __launch_bounds__(kFinishThreads)
@@ -331,15 +342,28 @@ cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream) {
   if (a.n <= kSmallRows) {
     int blocks = 1;
     while (blocks < 8 && blocks * 32 < a.n) blocks <<= 1;       // 32 rows per block until 8 blocks
-    int L = 32;
-    while (L > 1 && a.n * L > blocks * kSmallThreads) L >>= 1;
+    // 512-thread blocks fit on an SM beside a CTA of the tensor-core projection kernel, so they
+    // are resident (waiting) before it ends and do not keep the next call's CTAs off their SMs;
+    // they are used whenever a lane group still owns few enough partials for the one-pass fold.
+    auto lanes_for = [&](int threads) {
+      int l = 32;
+      while (l > 1 && a.n * l > blocks * threads) l >>= 1;
+      return l;
+    };
+    int threads = kSmallThreads;
+    if ((a.chunks + lanes_for(512) - 1) / lanes_for(512) <= kPerLane) threads = 512;
+    if (const char* env = getenv("TLR_FINISH_THREADS")) {   // tuning switch
+      const int e = atoi(env);
+      if (e == 256 || e == 512 || e == 1024) threads = e;
+    }
+    const int L = lanes_for(threads);
     attr[1].id = cudaLaunchAttributeClusterDimension;
     attr[1].val.clusterDim.x = static_cast<unsigned>(blocks);
     attr[1].val.clusterDim.y = 1;
     attr[1].val.clusterDim.z = 1;
     cfg.numAttrs = 2;
     cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
-    cfg.blockDim = dim3(kSmallThreads, 1, 1);
+    cfg.blockDim = dim3(static_cast<unsigned>(threads), 1, 1);
     return cudaLaunchKernelEx(&cfg, finish_small_kernel, a, L);
   }
   const int blocks = (a.n + kFinishWarps - 1) / kFinishWarps;
