@@ -200,10 +200,13 @@ tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t sha
                             int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream);
 
 /*
- * tlr_route_host -- the same step with HOST buffers: copies h to the device, runs
- * tlr_route, brings the six results back in one copy to a pinned buffer of the context,
- * synchronises the stream and hands them out to the caller's buffers.  Host buffers may
- * be pageable or pinned (a pinned h is faster).  Not reentrant on one context.  Output
+ * tlr_route_host -- the same step with HOST buffers: brings h to the device, runs
+ * tlr_route with the six results written straight into a pinned, device-visible buffer of
+ * the context, synchronises the stream and hands them out to the caller's buffers.  Host
+ * buffers may be pageable or pinned.  A pinned (or registered), 16-byte aligned h of up to
+ * 4 MB is fetched by a copy kernel rather than the copy engine, so that the projection
+ * kernel is launched, and streams W, while h is still on its way; anything else goes
+ * through cudaMemcpyAsync.  Not reentrant on one context.  Output
  * pointers may be NULL to skip that copy, except routed_count_host.  routed_idx_host
  * needs capacity n; only the first *routed_count_host entries are written.
  * Same errors as tlr_route, plus TLR_ERR_DEVICE_STATUS when a kernel raised

@@ -88,7 +88,8 @@ struct tlr_ctx {
   // them all to a pinned host mirror: token[n] conf[n] entropy[n] routed_idx[n] count mask[n].
   void* h_stage = nullptr;
   unsigned char* out_stage = nullptr;    // device, 17 * max_n + 8 bytes
-  unsigned char* out_pinned = nullptr;   // pinned host mirror of the same size, + 4 bytes for the status word
+  unsigned char* out_pinned = nullptr;   // pinned host mirror of the same size, + an aligned 4-byte status word
+  unsigned char* out_mapped = nullptr;   // the mirror as the device sees it (kernels write the results into it), or null
 
   // learned router (tlr_set_router_mlp)
   int mlp_hidden = 0;
@@ -228,6 +229,11 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
 
 }  // namespace
 
+static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, const tlr_route_options* opt,
+                             int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
+                             int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream,
+                             uint32_t* status_copy);
+
 extern "C" {
 
 const char* tlr_status_string(tlr_status s) {
@@ -273,11 +279,15 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
   ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
   ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
-  ok = ok && cudaMallocHost(&c->out_pinned, np * 17 + 8 + 4) == cudaSuccess;
+  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_all(c);
     return TLR_ERR_NOMEM;
+  }
+  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
+    cudaGetLastError();
+    c->out_mapped = nullptr;   // tlr_route_host then stages the outputs in device memory and copies them
   }
   if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
       cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
@@ -403,6 +413,17 @@ tlr_status tlr_route(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau,
 tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, const tlr_route_options* opt,
                         int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
                         int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream) {
+  return route_step(ctx, h_bf16_dev, n, tau, opt, token_dev, conf_dev, entropy_dev, route_mask_dev, routed_idx_dev,
+                    routed_count_dev, cuda_stream, nullptr);
+}
+
+}  // extern "C"
+
+// One routing step; status_copy (optional, device-visible) receives the status word after the last row.
+static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float tau, const tlr_route_options* opt,
+                             int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
+                             int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream,
+                             uint32_t* status_copy) {
   if (ctx == nullptr || n < 0 || routed_count_dev == nullptr) return TLR_ERR_ARG;
   if (opt != nullptr && opt->seq_len > 0 && (n % opt->seq_len != 0 || opt->first_routed_dev == nullptr))
     return TLR_ERR_ARG;
@@ -463,9 +484,12 @@ tlr_status tlr_route_ex(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, float t
   f.routed_count = routed_count_dev;
   f.ticket = ctx->ticket;
   f.status = ctx->status;
+  f.status_copy = status_copy;
   if (tlr::launch_finish(f, stream) != cudaSuccess) return TLR_ERR_CUDA;
   return TLR_OK;
 }
+
+extern "C" {
 
 tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, int32_t v_offset, void* summary_dev,
                              void* cuda_stream) {
@@ -528,24 +552,44 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
   if (n > 0 && h_bf16_host == nullptr) return TLR_ERR_ARG;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t nn = static_cast<size_t>(n);
-  if (n > 0 &&
-      cudaMemcpyAsync(ctx->h_stage, h_bf16_host, nn * ctx->d * 2, cudaMemcpyHostToDevice, stream) != cudaSuccess)
-    return TLR_ERR_CUDA;
+  if (n > 0) {
+    // h comes in by a copy kernel when the GPU can read the caller's buffer directly (pinned or
+    // registered host memory): the projection kernel is then launched while h is still on its way
+    // (see tlr_hostio.cu).  Pageable memory goes through the copy engine.
+    const size_t bytes = nn * ctx->d * 2;
+    cudaPointerAttributes attr;
+    const void* mapped = nullptr;
+    // Above a few MB the copy engine is faster than the copy kernel and there is nothing left to hide.
+    if (bytes <= (4u << 20) && (bytes & 15u) == 0 && (reinterpret_cast<uintptr_t>(h_bf16_host) & 15u) == 0 &&
+        cudaPointerGetAttributes(&attr, h_bf16_host) == cudaSuccess && attr.type == cudaMemoryTypeHost)
+      mapped = attr.devicePointer;
+    cudaGetLastError();
+    if (mapped != nullptr) {
+      if (tlr::launch_host_copy(mapped, ctx->h_stage, bytes, stream) != cudaSuccess) return TLR_ERR_CUDA;
+    } else if (cudaMemcpyAsync(ctx->h_stage, h_bf16_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+      return TLR_ERR_CUDA;
+    }
+  }
   // layout of the output block for this n (all offsets are multiples of 4)
   const size_t off_conf = 4 * nn, off_ent = 8 * nn, off_idx = 12 * nn, off_count = 16 * nn, off_mask = 16 * nn + 4;
   const size_t out_bytes = 17 * nn + 4;
-  unsigned char* dev = ctx->out_stage;
-  const tlr_status st = tlr_route(ctx, ctx->h_stage, n, tau, reinterpret_cast<int32_t*>(dev),
-                                  reinterpret_cast<float*>(dev + off_conf), reinterpret_cast<float*>(dev + off_ent),
-                                  dev + off_mask, reinterpret_cast<int32_t*>(dev + off_idx),
-                                  reinterpret_cast<int32_t*>(dev + off_count), cuda_stream);
-  if (st != TLR_OK) return st;
   unsigned char* pin = ctx->out_pinned;
-  uint32_t* pin_status = reinterpret_cast<uint32_t*>(pin + static_cast<size_t>(ctx->max_n) * 17 + 8);
-  if (cudaMemcpyAsync(pin, dev, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaMemcpyAsync(pin_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
-      cudaStreamSynchronize(stream) != cudaSuccess)
+  const size_t off_status = (static_cast<size_t>(ctx->max_n) * 17 + 8 + 3) & ~static_cast<size_t>(3);   // a 4-byte word
+  uint32_t* pin_status = reinterpret_cast<uint32_t*>(pin + off_status);
+  // The kernels write the six outputs and the status word straight into the pinned host block
+  // (4 KB at n = 256); without a device view of it they go to device memory and are copied.
+  const bool direct = ctx->out_mapped != nullptr;
+  unsigned char* dev = direct ? ctx->out_mapped : ctx->out_stage;
+  const tlr_status st = route_step(ctx, ctx->h_stage, n, tau, nullptr, reinterpret_cast<int32_t*>(dev),
+                                   reinterpret_cast<float*>(dev + off_conf), reinterpret_cast<float*>(dev + off_ent),
+                                   dev + off_mask, reinterpret_cast<int32_t*>(dev + off_idx),
+                                   reinterpret_cast<int32_t*>(dev + off_count), cuda_stream,
+                                   direct ? reinterpret_cast<uint32_t*>(dev + off_status) : nullptr);
+  if (st != TLR_OK) return st;
+  if (!direct && (cudaMemcpyAsync(pin, dev, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+                  cudaMemcpyAsync(pin_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess))
     return TLR_ERR_CUDA;
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return TLR_ERR_CUDA;
   int32_t count = 0;
   memcpy(&count, pin + off_count, 4);
   *routed_count_host = count;

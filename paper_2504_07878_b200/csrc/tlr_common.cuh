@@ -109,6 +109,7 @@ struct FinishLaunch {
   int32_t* routed_count;
   unsigned int* ticket;     // zero before the launch; the kernel leaves it zero again
   uint32_t* status;
+  uint32_t* status_copy;    // optional: receives the status word once every row is scored (host-mapped memory)
 };
 cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
 
@@ -117,6 +118,10 @@ cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
 cudaError_t launch_shard_summary(const Partial* partials, int n, int chunks, int v_offset, Partial* summary,
                                  cudaStream_t stream);
 cudaError_t launch_shard_gather(const Partial* gathered, int shards, int n, Partial* partials, cudaStream_t stream);
+
+// Copy of `bytes` (a multiple of 16) from host memory the device can read directly to device
+// memory, done by a kernel so that the projection kernel behind it can be launched early.
+cudaError_t launch_host_copy(const void* src_mapped, void* dst, size_t bytes, cudaStream_t stream);
 
 struct MlpLaunch {
   const void* h;        // bf16 [n][d]

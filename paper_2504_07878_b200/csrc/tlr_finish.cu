@@ -272,7 +272,10 @@ finish_small_kernel(const FinishLaunch a, const int L) {
     base_out += total;
     __syncthreads();
   }
-  if (threadIdx.x == 0) *a.routed_count = base_out;
+  if (threadIdx.x == 0) {
+    *a.routed_count = base_out;
+    if (a.status_copy != nullptr) *a.status_copy = atomicOr(a.status, 0u);   // every row has been scored by now
+  }
 }
 
 __global__ void __launch_bounds__(kFinishThreads)
@@ -325,6 +328,7 @@ finish_kernel(const FinishLaunch a) {
   }
   if (threadIdx.x == 0) {
     *a.routed_count = base_out;
+    if (a.status_copy != nullptr) *a.status_copy = atomicOr(a.status, 0u);
     *a.ticket = 0u;  // ready for the next call on this context
   }
 }

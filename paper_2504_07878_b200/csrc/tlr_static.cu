@@ -175,7 +175,7 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
     }
   }
 
-  tlr::FinishLaunch f;
+  tlr::FinishLaunch f = {};
   f.partials = partials;
   f.n = n;
   f.chunks = chunks;

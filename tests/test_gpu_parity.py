@@ -162,22 +162,37 @@ def test_two_runs_bit_identical_and_paths_agree(pkg):
     np.testing.assert_allclose(a["conf"], c["conf"], rtol=1e-3)
 
 
-def test_host_buffer_entry_point(pkg):
-    W, hid = small_case(100, 128, 6000, seed=6, planted=0.1)
-    ref = O.route_oracle(S.bf16_bits(hid.h), S.bf16_bits(W), 0.5)
+@pytest.mark.parametrize("how,n,d,V", [("pinned", 100, 128, 6000),      # h fetched by the copy kernel
+                                       ("pageable", 100, 128, 6000),    # h through the copy engine
+                                       ("pinned", 300, 896, 3001),      # pair kernel behind the copy kernel
+                                       ("pinned", 2500, 896, 2048),     # more than 4 MB of h: copy engine again
+                                       ("pinned", 37, 64, 999),         # odd max_n: the status word's alignment
+                                       ("pinned", 0, 128, 6000)])
+def test_host_buffer_entry_point(pkg, how, n, d, V):
+    W, hid = small_case(max(n, 1), d, V, seed=6, planted=0.1)
+    hrows = hid.h[:n]
     Wd = W.cuda()
-    ctx = pkg.tlr_create(128, 6000, Wd, 128)
-    n = 100
-    h = hid.h.pin_memory()
-    token = torch.empty(n, dtype=torch.int32).pin_memory(); conf = torch.empty(n).pin_memory()
-    ent = torch.empty(n).pin_memory(); mask = torch.empty(n, dtype=torch.uint8).pin_memory()
-    idx = torch.full((n,), -1, dtype=torch.int32).pin_memory(); cnt = torch.zeros(1, dtype=torch.int32).pin_memory()
-    pkg.tlr_route_host(ctx, h, n, 0.5, token, conf, ent, mask, idx, cnt)
-    gpu = {"token": token.numpy(), "conf": conf.numpy(), "entropy": ent.numpy(), "route_mask": mask.numpy(),
-           "routed_idx": idx.numpy(), "routed_count": int(cnt.item())}
-    check_against_oracle(ref, gpu)
-    check_self_consistency(gpu, 0.5, 6000)
-    assert gpu["routed_count"] == ref.routed_count
+    ctx = pkg.tlr_create(d, V, Wd, max(n, 1) + 28)
+    pin = (lambda x: x.pin_memory()) if how == "pinned" else (lambda x: x)
+    h = pin(hrows.contiguous())
+    m = max(n, 1)
+    token = pin(torch.empty(m, dtype=torch.int32)); conf = pin(torch.empty(m))
+    ent = pin(torch.empty(m)); mask = pin(torch.empty(m, dtype=torch.uint8))
+    idx = pin(torch.full((m,), -1, dtype=torch.int32)); cnt = pin(torch.full((1,), -9, dtype=torch.int32))
+    for _ in range(2):                                  # twice: the context's staging is reused
+        pkg.tlr_route_host(ctx, h, n, 0.5, token, conf, ent, mask, idx, cnt)
+    if n == 0:
+        assert int(cnt.item()) == 0
+        pkg.tlr_destroy(ctx)
+        return
+    ref = O.route_oracle(S.bf16_bits(hrows), S.bf16_bits(W), 0.5)
+    gpu = {"token": token.numpy()[:n], "conf": conf.numpy()[:n], "entropy": ent.numpy()[:n],
+           "route_mask": mask.numpy()[:n], "routed_idx": idx.numpy(), "routed_count": int(cnt.item())}
+    rep = check_against_oracle(ref, gpu)
+    check_self_consistency(gpu, 0.5, V)
+    if rep["route_exempt_rows"] == 0:
+        assert gpu["routed_count"] == ref.routed_count
+    assert pkg.tlr_last_device_status(ctx) == 0
     pkg.tlr_destroy(ctx)
 
 
