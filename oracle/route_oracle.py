@@ -22,6 +22,8 @@ What it computes, per decoding position i (one row of ``h``):
   Variants of steps 5-6: one threshold per row, the opposite polarity (Sec. 2.2:
   defer when the score exceeds the threshold), and the first routed position of
   every sequence (Sec. 4.1: where the re-processing of a returned context stops).
+  8-bit copy of W (decode batches): e4m3 codes and one scale per row; the step is
+  defined as the step on the de-quantised matrix (dequantize_e4m3).
   Vocabulary-sharded form (several GPUs, each a contiguous range of W's rows):
   shard_summary is what one range reports per row, merge_summaries combines the
   ranges; together they must reproduce steps 2-4 (pinned against them).
@@ -164,6 +166,25 @@ def with_threshold(result: RouteResult, tau, route_above: bool = False) -> Route
     """The same per-row scores with steps 5-6 redone for another threshold or polarity."""
     mask, idx, count, tau32 = route_decision(result.conf, tau, route_above)
     return RouteResult(result.token, result.conf, result.entropy, mask, idx, count, result.top2_gap, tau32)
+
+
+def e4m3_value(codes: np.ndarray) -> np.ndarray:
+    """Values of OCP 8-bit floats "e4m3": bit 7 sign, bits 6..3 exponent E (bias 7), bits 2..0
+    mantissa M.  E = 0: (M/8) * 2^-6 (subnormal);  otherwise (1 + M/8) * 2^(E-7); there are no
+    infinities and E = 15 with M = 7 (0x7f, 0xff) is NaN.  fp64 out."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    E = (c >> 3) & 15
+    M = (c & 7).astype(np.float64)
+    mag = np.where(E == 0, (M / 8.0) * 2.0 ** -6, (1.0 + M / 8.0) * np.exp2((E - 7).astype(np.float64)))
+    mag = np.where((E == 15) & ((c & 7) == 7), np.nan, mag)
+    return np.where(c & 0x80, -mag, mag)
+
+
+def dequantize_e4m3(codes: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """The LM head an 8-bit copy stands for: W[v][k] = scale[v] * e4m3_value(codes[v][k]), fp64.
+    The routing step on an 8-bit W is, by definition, the step on this matrix (route_oracle with
+    W64 = dequantize_e4m3(...)); the hidden states stay bf16."""
+    return e4m3_value(codes) * np.asarray(scale, dtype=np.float64)[:, None]
 
 
 def shard_summary(h_bits: np.ndarray, W_shard_bits: np.ndarray, v_offset: int):

@@ -54,6 +54,8 @@ def load_library() -> ctypes.CDLL:
     lib = ctypes.CDLL(LIB_PATH)
     P = c_void_p
     lib.tlr_create.argtypes = [c_int32, c_int32, P, c_int32, POINTER(P)]
+    lib.tlr_create_fp8.argtypes = [c_int32, c_int32, P, P, c_int32, POINTER(P)]
+    lib.tlr_create_fp8.restype = c_int32
     lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_route_ex.argtypes = [P, P, c_int32, c_float, POINTER(TlrRouteOptions), P, P, P, P, P, P, P]
     lib.tlr_route_ex.restype = c_int32
@@ -114,6 +116,13 @@ def tlr_create(d: int, V: int, W, max_n: int) -> c_void_p:
     """W: CUDA bf16 [V, d] contiguous tensor (or a raw device address).  It is borrowed, not copied."""
     ctx = c_void_p(0)
     _check(load_library().tlr_create(d, V, _ptr(W), max_n, byref(ctx)), "tlr_create")
+    return ctx
+
+
+def tlr_create_fp8(d: int, V: int, W_e4m3, wscale, max_n: int) -> c_void_p:
+    """W_e4m3: CUDA uint8 (or float8_e4m3fn) [V, d] codes, wscale: CUDA float32 [V]; both borrowed.  Decode batches only."""
+    ctx = c_void_p(0)
+    _check(load_library().tlr_create_fp8(d, V, _ptr(W_e4m3), _ptr(wscale), max_n, byref(ctx)), "tlr_create_fp8")
     return ctx
 
 
@@ -225,14 +234,21 @@ def tlr_read_kernel_timing(ctx):
 class Router:
     """Convenience owner of a context and its output tensors (allocation only; no arithmetic)."""
 
-    def __init__(self, W: torch.Tensor, max_n: int):
-        if not (W.is_cuda and W.dtype == torch.bfloat16 and W.dim() == 2 and W.is_contiguous()):
-            raise ValueError("W must be a contiguous CUDA bf16 [V, d] tensor")
+    def __init__(self, W: torch.Tensor, max_n: int, wscale: torch.Tensor = None):
+        """W: bf16 [V, d]; or, with wscale (float32 [V]), e4m3 codes (uint8 / float8_e4m3fn) [V, d] for decode batches."""
+        fp8 = wscale is not None
+        ok_dtype = W.dtype in (torch.uint8, torch.float8_e4m3fn) if fp8 else W.dtype == torch.bfloat16
+        if not (W.is_cuda and ok_dtype and W.dim() == 2 and W.is_contiguous()):
+            raise ValueError("W must be a contiguous CUDA [V, d] tensor, bf16 or (with wscale) e4m3 codes")
+        if fp8 and not (wscale.is_cuda and wscale.dtype == torch.float32 and wscale.shape == (W.shape[0],)
+                        and wscale.is_contiguous()):
+            raise ValueError("wscale must be a contiguous CUDA float32 [V] tensor")
         self.W = W                      # keep the borrowed matrix alive
+        self.wscale = wscale
         self.V, self.d = W.shape
         self.max_n = max_n
         with torch.cuda.device(W.device):
-            self.ctx = tlr_create(self.d, self.V, W, max_n)
+            self.ctx = tlr_create_fp8(self.d, self.V, W, wscale, max_n) if fp8 else tlr_create(self.d, self.V, W, max_n)
             dev = W.device
             self.token = torch.empty(max_n, dtype=torch.int32, device=dev)
             self.conf = torch.empty(max_n, dtype=torch.float32, device=dev)

@@ -100,6 +100,12 @@ struct tlr_ctx {
   float* mlp_scores = nullptr;     // [max_n][hidden blocks] partial sums of the output layer
   int mlp_blocks_cap = 0;
 
+  // fp8 copy of W (tlr_create_fp8): e4m3 codes, one scale per row; h is split into two e4m3 parts per call
+  bool fp8 = false;
+  const float* wscale = nullptr;
+  uint8_t* h_parts = nullptr;     // [2][tc8_max_rows()][d]
+  float* hscale = nullptr;        // [tc8_max_rows()]
+
   // test hook (tlr_debug_inject)
   int debug_kind = 0;
   unsigned long long debug_wait_ns = 0;
@@ -110,6 +116,18 @@ struct tlr_ctx {
 };
 
 namespace {
+
+// Rows of `cols` e4m3 bytes, boxes of 128 bytes x box_rows, 128-byte swizzle.
+bool make_map8(tlr_ctx* c, CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(cols)};
+  const cuuint32_t box[2] = {128u, static_cast<cuuint32_t>(box_rows)};
+  const cuuint32_t elem[2] = {1u, 1u};
+  const CUresult r = c->encode(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box,
+                               elem, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                               CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
 
 bool make_map(tlr_ctx* c, CUtensorMap* map, const void* base, int rows, int cols, int box_rows) {
   const cuuint64_t dims[2] = {static_cast<cuuint64_t>(cols), static_cast<cuuint64_t>(rows)};
@@ -132,7 +150,18 @@ void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
   out->path = path;
   out->launches = n > 0 ? 2 : 1;
   out->reserved = 0;
-  if (path == TLR_PATH_TC) {
+  if (c->fp8) {
+    tlr::Tc8Config cfg;
+    tlr::TcPlan tp;
+    tlr::tc8_configure(n, &cfg);
+    tlr::tc_plan(n <= 128 ? n : 128, c->V, 1, c->sm_count, tlr::kMaxChunks, &tp);
+    out->vocab_chunks = tp.chunks;
+    out->row_units = 1;
+    out->grid = tp.chunks < c->sm_count ? tp.chunks : c->sm_count;
+    out->block = tlr::tc8_threads();
+    out->smem_bytes = cfg.smem_bytes;
+    out->launches = n > 0 ? 3 : 1;
+  } else if (path == TLR_PATH_TC) {
     tlr::TcConfig cfg;
     tlr::TcPlan tp;
     tlr::tc_configure(n, &cfg);
@@ -164,6 +193,8 @@ void free_all(tlr_ctx* c) {
   cudaFree(c->out_stage);
   cudaFreeHost(c->out_pinned);
   cudaFree(c->mlp_scores);
+  cudaFree(c->h_parts);
+  cudaFree(c->hscale);
   for (cudaEvent_t e : c->events) cudaEventDestroy(e);
   delete c;
 }
@@ -183,7 +214,34 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
     if (cudaEventRecord(ev0, stream) != cudaSuccess) return TLR_ERR_CUDA;
   }
   cudaError_t e;
-  if (plan.path == TLR_PATH_TC) {
+  if (ctx->fp8) {
+    tlr::Tc8Config cfg;
+    tlr::TcPlan tp;
+    tlr::tc8_configure(n, &cfg);
+    tlr::tc_plan(n, ctx->V, 1, ctx->sm_count, tlr::kMaxChunks, &tp);
+    if (tlr::launch_h_split(h_bf16_dev, n, ctx->d, cfg.a_rows, ctx->h_parts, ctx->hscale, stream) != cudaSuccess)
+      return TLR_ERR_CUDA;
+    CUtensorMap map_h;
+    if (!make_map8(ctx, &map_h, ctx->h_parts, 2 * cfg.a_rows, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
+    tlr::Tc8Params p = {};
+    p.n = n;
+    p.d = ctx->d;
+    p.V = ctx->V;
+    p.chunks = tp.chunks;
+    p.granules = tp.granules;
+    p.tiles_per_unit = tp.tiles_per_unit;
+    p.granule_rows = tp.granule_rows;
+    p.a_rows = cfg.a_rows;
+    p.a_stages = cfg.a_stages;
+    p.b_stages = cfg.b_stages;
+    p.wait_limit_ns = ctx->debug_wait_ns;
+    p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
+    p.hscale = ctx->hscale;
+    p.wscale = ctx->wscale;
+    p.partials = ctx->partials;
+    p.status = ctx->status;
+    e = tlr::launch_tc8_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid, stream);
+  } else if (plan.path == TLR_PATH_TC) {
     tlr::TcConfig cfg;
     tlr::TcPlan tp;
     tlr::tc_configure(n, &cfg);
@@ -318,6 +376,73 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
   return TLR_OK;
 }
 
+tlr_status tlr_create_fp8(int32_t d, int32_t V, const void* W_e4m3_dev, const float* wscale_dev, int32_t max_n,
+                          tlr_ctx** out) {
+  if (out == nullptr) return TLR_ERR_ARG;
+  *out = nullptr;
+  if (d <= 0 || V <= 0 || max_n <= 0 || W_e4m3_dev == nullptr || wscale_dev == nullptr) return TLR_ERR_ARG;
+  if ((reinterpret_cast<uintptr_t>(W_e4m3_dev) & 15u) != 0 || (reinterpret_cast<uintptr_t>(wscale_dev) & 3u) != 0)
+    return TLR_ERR_ALIGN;
+  if (d % 16 != 0) return TLR_ERR_UNSUPPORTED;         // rows of 8-bit W must be multiples of 16 bytes for TMA
+  if (static_cast<long long>(V) + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TLR_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TLR_ERR_CUDA;
+  if (prop.major != 10) return TLR_ERR_UNSUPPORTED;
+  tlr_ctx* c = new (std::nothrow) tlr_ctx();
+  if (c == nullptr) return TLR_ERR_NOMEM;
+  c->device = dev;
+  c->sm_count = prop.multiProcessorCount;
+  c->d = d;
+  c->V = V;
+  c->max_n = max_n;
+  c->W = W_e4m3_dev;
+  c->wscale = wscale_dev;
+  c->fp8 = true;
+  const size_t np = static_cast<size_t>(max_n);
+  const size_t rows8 = static_cast<size_t>(tlr::tc8_max_rows());
+  bool ok = true;
+  ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
+  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->h_parts, 2 * rows8 * d) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->hscale, rows8 * sizeof(float)) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_all(c);
+    return TLR_ERR_NOMEM;
+  }
+  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
+    cudaGetLastError();
+    c->out_mapped = nullptr;
+  }
+  if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
+      cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
+    free_all(c);
+    return TLR_ERR_CUDA;
+  }
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess && fn != nullptr) {
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+    if (make_map8(c, &c->map_w128, W_e4m3_dev, V, d, 128) && make_map8(c, &c->map_w64, W_e4m3_dev, V, d, 64) &&
+        make_map8(c, &c->map_w16, W_e4m3_dev, V, d, 16) && tlr::tc8_prepare() == cudaSuccess)
+      c->tc_ok = true;
+  }
+  cudaGetLastError();
+  if (!c->tc_ok) {
+    free_all(c);
+    return TLR_ERR_CUDA;
+  }
+  *out = c;
+  return TLR_OK;
+}
+
 tlr_status tlr_destroy(tlr_ctx* ctx) {
   if (ctx == nullptr) return TLR_OK;
   free_all(ctx);
@@ -392,6 +517,7 @@ tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path) {
   if (ctx == nullptr) return TLR_ERR_ARG;
   if (path != TLR_PATH_AUTO && path != TLR_PATH_SIMT && path != TLR_PATH_TC) return TLR_ERR_ARG;
   if (path == TLR_PATH_TC && !ctx->tc_ok) return TLR_ERR_UNSUPPORTED;
+  if (path == TLR_PATH_SIMT && ctx->fp8) return TLR_ERR_UNSUPPORTED;
   ctx->forced = path;
   return TLR_OK;
 }
@@ -432,6 +558,7 @@ static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, fl
   if (opt != nullptr && opt->score_source != TLR_SCORE_CONF && opt->score_source != TLR_SCORE_MLP) return TLR_ERR_ARG;
   if (want_mlp && ctx->mlp_hidden == 0) return TLR_ERR_ARG;
   if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (ctx->fp8 && n > tlr::tc8_max_rows()) return TLR_ERR_UNSUPPORTED;   // the fp8 copy serves decode batches only
   if (n > 0) {
     if (h_bf16_dev == nullptr || token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr ||
         route_mask_dev == nullptr || routed_idx_dev == nullptr)
@@ -500,6 +627,7 @@ tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, in
   if ((reinterpret_cast<uintptr_t>(h_bf16_dev) & 15u) != 0 || (reinterpret_cast<uintptr_t>(summary_dev) & 15u) != 0)
     return TLR_ERR_ALIGN;
   if (static_cast<long long>(v_offset) + ctx->V + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+  if (ctx->fp8 && n > tlr::tc8_max_rows()) return TLR_ERR_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   tlr_plan plan;
   fill_plan(ctx, n, &plan);

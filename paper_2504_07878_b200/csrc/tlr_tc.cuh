@@ -36,6 +36,37 @@ struct TcParams {
   uint32_t* status;
 };
 
+// ---- fp8-W decode kernel (tlr_tc8.cu): one CTA per worker, n <= tc8_max_rows()
+struct Tc8Config {
+  int a_rows;       // rows of an h slab part held in shared memory (16..64)
+  int a_stages;     // depth of the h ring (a stage = both parts of one 128-wide slab)
+  int b_stages;     // depth of the W ring (a stage = up to 256 rows x 128 bytes)
+  int smem_bytes;
+};
+
+struct Tc8Params {
+  int n, d, V;
+  int chunks, granules, tiles_per_unit, granule_rows;
+  int a_rows, a_stages, b_stages;
+  unsigned long long wait_limit_ns;
+  int debug_drop_w_copies;
+  const float* hscale;   // [n] power-of-two scale of every row of h (written by the split kernel)
+  const float* wscale;   // [V] scale of every row of W
+  Partial* partials;     // [n][chunks]
+  uint32_t* status;
+};
+
+int tc8_threads();
+int tc8_max_rows();
+void tc8_configure(int n, Tc8Config* c);
+cudaError_t tc8_prepare();
+// h [n][d] bf16 -> parts [2][rows_alloc][d] e4m3 (rows n.. zero) and hscale[n]
+cudaError_t launch_h_split(const void* h_bf16, int n, int d, int rows_alloc, uint8_t* parts, float* hscale,
+                           cudaStream_t stream);
+cudaError_t launch_tc8_projection(const CUtensorMap& map_h, const CUtensorMap& map_w128, const CUtensorMap& map_w64,
+                                  const CUtensorMap& map_w16, const Tc8Params& p, const Tc8Config& c, int workers,
+                                  cudaStream_t stream);
+
 int tc_threads();
 int tc_enumerate_tiles(const TcParams& p, int cta, int workers, int* out, int capacity);
 void tc_configure(int n, TcConfig* c);

@@ -367,3 +367,32 @@ def test_shard_summary_hand_worked():
     assert token[0] == 1 and conf[0] == pytest.approx(1 / Ssum)
     p = np.array([math.exp(-2), 1.0, 1.0, math.exp(-1)]) / Ssum
     assert ent[0] == pytest.approx(float(-(p * np.log(p)).sum()))
+
+
+# ---------------------------------------------------------------- 8-bit copy of W
+
+def test_e4m3_values_against_the_format_definition():
+    """Hand-picked codes of the OCP e4m3 format, its extremes, its symmetry and its ordering."""
+    v = O.e4m3_value(np.arange(256, dtype=np.uint8))
+    assert v[0x00] == 0.0 and v[0x80] == 0.0
+    assert v[0x01] == 2.0 ** -9 and v[0x07] == 7 * 2.0 ** -9          # subnormals
+    assert v[0x08] == 2.0 ** -6                                        # smallest normal
+    assert v[0x38] == 1.0 and v[0x3c] == 1.5 and v[0x40] == 2.0 and v[0xc0] == -2.0
+    assert v[0x7e] == 448.0 and v[0xfe] == -448.0                      # largest finite
+    assert np.isnan(v[0x7f]) and np.isnan(v[0xff])
+    assert np.all(np.diff(v[:0x7f]) > 0)                               # magnitudes grow with the code
+    assert np.array_equal(v[0x80:0xff], -v[0x00:0x7f])
+    import torch as _t                                                  # a library's decoder of the same format
+    lib = _t.arange(256, dtype=_t.uint8).view(_t.float8_e4m3fn).double().numpy()
+    assert np.array_equal(np.nan_to_num(v, nan=-1.0), np.nan_to_num(lib, nan=-1.0))
+
+
+def test_dequantized_head_and_generator_recipe():
+    codes, scale = S.make_W8(32, 50, seed=3, std=0.02)
+    W = O.dequantize_e4m3(codes.numpy(), scale.numpy())
+    assert W.shape == (50, 32) and np.all(np.isfinite(W))
+    assert np.allclose(np.abs(W).max(axis=1), 448.0 * scale.numpy().astype(np.float64), rtol=1e-6)   # row maximum maps to 448
+    assert 0.015 < W.std() < 0.025                                     # still the N(0, 0.02^2) head
+    # a hand-made head: codes 0x38 (1.0) and 0xc0 (-2.0) with scales 0.5 and 3
+    hand = O.dequantize_e4m3(np.array([[0x38, 0xc0], [0x40, 0x01]], np.uint8), np.array([0.5, 3.0], np.float32))
+    assert np.array_equal(hand, np.array([[0.5, -1.0], [6.0, 3.0 * 2.0 ** -9]]))

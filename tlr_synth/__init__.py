@@ -113,3 +113,44 @@ def bf16_from_values(values) -> torch.Tensor:
     if not torch.equal(b.double(), t):
         raise ValueError("values are not exactly representable in bf16")
     return b
+
+
+# ---------------------------------------------------------------- 8-bit copy of W (decode batches)
+
+def _e4m3_magnitudes() -> np.ndarray:
+    """The 127 finite magnitudes of the OCP e4m3 format in code order (code 0..126): 1 sign bit,
+    4 exponent bits (bias 7), 3 mantissa bits; exponent 0 is subnormal (m/8 * 2^-6); no infinities,
+    and code 127 (0x7f) is NaN, so the largest finite magnitude is 448.  Used here only to CHOOSE
+    codes; what the codes mean to the routing step is defined by the callee."""
+    out = np.empty(127, np.float64)
+    for c in range(127):
+        e, m = c >> 3, c & 7
+        out[c] = (m / 8.0) * 2.0 ** -6 if e == 0 else (1.0 + m / 8.0) * 2.0 ** (e - 7)
+    return out
+
+
+def make_W8(d: int, V: int, seed: int = 0, std: float = 0.02):
+    """An 8-bit LM head: (codes uint8 [V, d], scale float32 [V]) with W[v][k] = scale[v] * e4m3(codes[v][k]).
+
+    Recipe: the same N(0, std^2) draw as make_W (in fp32, not rounded to bf16), one scale per row
+    that maps the row's largest magnitude to 448, and for every element the nearest e4m3 code of
+    value / scale (ties to the even code)."""
+    g = _gen(seed, _STREAM_W)
+    mags = _e4m3_magnitudes()
+    mid = (mags[1:] + mags[:-1]) / 2.0
+    codes = np.empty((V, d), np.uint8)
+    scale = np.empty(V, np.float32)
+    rows_per_chunk = max(1, (1 << 22) // max(d, 1))
+    for r0 in range(0, V, rows_per_chunk):
+        r1 = min(V, r0 + rows_per_chunk)
+        w = (torch.randn((r1 - r0, d), generator=g, dtype=torch.float32) * std).numpy().astype(np.float64)
+        amax = np.abs(w).max(axis=1)
+        s = np.where(amax > 0, amax / 448.0, 1.0).astype(np.float32)
+        x = w / s.astype(np.float64)[:, None]
+        a = np.minimum(np.abs(x), 448.0)
+        c = np.searchsorted(mid, a, side="left")                 # nearest magnitude; exact ties go down ...
+        tie = (c < 126) & (a == mid[np.minimum(c, 125)]) & (c % 2 == 1)
+        c = np.where(tie, c + 1, c)                               # ... unless the upper neighbour is the even code
+        codes[r0:r1] = (c.astype(np.uint8) | np.where(x < 0, 0x80, 0).astype(np.uint8))
+        scale[r0:r1] = s
+    return torch.from_numpy(codes), torch.from_numpy(scale)
