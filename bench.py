@@ -63,9 +63,10 @@ def measured_peaks():
     return dict(FALLBACK_PEAKS), "fallback"
 
 
-def algorithmic_bytes(n, d, V):
-    """W once + h once + the six outputs (17 bytes per row + the count)."""
-    return 2 * V * d + 2 * n * d + 17 * n + 4
+def algorithmic_bytes(n, d, V, fp8=False):
+    """W once + h once + the six outputs (17 bytes per row + the count); an 8-bit W is V*d bytes + V scales."""
+    w_bytes = V * d + 4 * V if fp8 else 2 * V * d
+    return w_bytes + 2 * n * d + 17 * n + 4
 
 
 def algorithmic_flops(n, d, V):
@@ -163,13 +164,24 @@ def run_ours(args):
     tau = 0.5 if wl.tau is None else wl.tau
     if args.tau is not None:
         tau = args.tau
-    W_host = S.make_W(d, V, seed=0)
-    hid = S.make_h(n, d, seed=rank, W=W_host, planted_fraction=wl.planted_fraction)
-    # two device copies of W, alternated step by step: together with W > L2 this makes every
-    # step stream W from HBM rather than from whatever the previous step left in L2
+    fp8 = bool(args.fp8)
+    if fp8 and n > 64:
+        raise SystemExit("--fp8 serves decode batches only (n <= 64): pick decode16 or sweep1/8/64")
+    # two device copies of W, alternated step by step: together with W > L2 (or, for the 8-bit copy
+    # of the 0.5B head, two copies > L2) this makes every step stream W from HBM rather than from
+    # whatever the previous step left in L2
     copies = 2
-    Ws = [W_host.cuda() for _ in range(copies)]
-    routers = [P.Router(w, max_n=n) for w in Ws]
+    if fp8:
+        codes, wscale = S.make_W8(d, V, seed=0)
+        W_host = None
+        hid = S.make_h(n, d, seed=rank)
+        Ws = [(codes.cuda(), wscale.cuda()) for _ in range(copies)]
+        routers = [P.Router(c, max_n=n, wscale=sc) for c, sc in Ws]
+    else:
+        W_host = S.make_W(d, V, seed=0)
+        hid = S.make_h(n, d, seed=rank, W=W_host, planted_fraction=wl.planted_fraction)
+        Ws = [W_host.cuda() for _ in range(copies)]
+        routers = [P.Router(w, max_n=n) for w in Ws]
     h_dev = hid.h.cuda()
     plan = P.tlr_plan_query(routers[0].ctx, n)
     stream = torch.cuda.current_stream()
@@ -268,31 +280,34 @@ def run_ours(args):
     value = job_throughput(world, n, ms_per_step * 1e-3)
     hbm_bound = n <= RIDGE_ROWS_HBM
     if hbm_bound:
-        achieved = algorithmic_bytes(n, d, V) / (kernel_ms * 1e-3) / 1e9
+        achieved = algorithmic_bytes(n, d, V, fp8) / (kernel_ms * 1e-3) / 1e9
         peak = float(peaks["hbm_gbs"])
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s"}
     else:
         achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
         peak = float(peaks.get("bf16_tflops_sustained" if ms_total > 1000 else "bf16_tflops", peaks["bf16_tflops"]))
         roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s"}
-    roof.update({"frac": achieved / peak, "traffic": ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V),
+    roof.update({"frac": achieved / peak, "traffic": None if fp8 else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
                  "peak_source": "of " + peak_kind,
-                 "kernel": "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel",
+                 "kernel": ("h_split_kernel + tc8_projection_kernel" if fp8 else
+                            "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel"),
                  "kernel_ms": kernel_ms, "kernel_launches_timed": launches,
                  "tensor_frac_same_launch": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
                  float(peaks["bf16_tflops"]),
-                 "hbm_frac_same_launch": algorithmic_bytes(n, d, V) / (kernel_ms * 1e-3) / 1e9 /
+                 "hbm_frac_same_launch": algorithmic_bytes(n, d, V, fp8) / (kernel_ms * 1e-3) / 1e9 /
                  float(peaks["hbm_gbs"])})
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
         "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-        "dtype": "bf16 in, fp32 accumulate and softmax statistics", "data": "synthetic",
-        "config": {"workload": "%s: n=%d rows, d=%d, V=%d, tau=%g%s" % (wl.name, n, d, V, tau,
+        "dtype": ("e4m3 W with one scale per row, bf16 h split into two e4m3 parts, fp32 accumulate and softmax statistics"
+                  if fp8 else "bf16 in, fp32 accumulate and softmax statistics"), "data": "synthetic",
+        "config": {"workload": "%s%s: n=%d rows, d=%d, V=%d, tau=%g%s" % (wl.name, " with an 8-bit copy of W" if fp8 else "",
+                                                                        n, d, V, tau,
                                                                        ", %.0f%% planted rows" % (100 * wl.planted_fraction)
                                                                        if wl.planted_fraction else ""),
                    "l2": "inputs larger than L2: W is %.0f MB and two device copies of it alternate between steps"
-                         % (2 * V * d / 1e6),
+                         % ((V * d if fp8 else 2 * V * d) / 1e6),
                    "path": int(plan.path), "grid": int(plan.grid), "block": int(plan.block),
                    "vocab_chunks": int(plan.vocab_chunks), "routed_rows_per_step": routed,
                    "variants": (("per-row tau + first routed per sequence of %d" % variant_args["seq_len"])
@@ -305,7 +320,7 @@ def run_ours(args):
         "roofline": roof,
     }
     if world == 1 and not args.no_cpu_baseline:
-        out["cpu_baseline"] = cpu_baseline(wl, W_host, hid, tau, budget_s=15.0)
+        out["cpu_baseline"] = cpu_baseline(wl, W_host, hid, tau, budget_s=15.0, w8=(codes, wscale) if fp8 else None)
     print(json.dumps(out))
 
 
@@ -320,11 +335,15 @@ def blas_threads():
     return os.cpu_count() or 1
 
 
-def cpu_baseline(wl, W_host, hid, tau, budget_s):
+def cpu_baseline(wl, W_host, hid, tau, budget_s, w8=None):
     """The fp64 oracle, as it stands, on a bounded sample of the workload's rows."""
     from oracle import route_oracle as O
-    Wb = S.bf16_bits(W_host)
-    W64 = O.bf16_bits_to_f64(Wb)
+    if w8 is not None:                       # the 8-bit head: the oracle runs on the de-quantised matrix
+        Wb = None
+        W64 = O.dequantize_e4m3(w8[0].numpy(), w8[1].numpy())
+    else:
+        Wb = S.bf16_bits(W_host)
+        W64 = O.bf16_bits_to_f64(Wb)
     hb = S.bf16_bits(hid.h)
     probe = min(8, wl.n)
     t0 = time.perf_counter()
@@ -390,6 +409,9 @@ def main():
                     help="route with per-row thresholds and report the first routed position per sequence "
                          "(tlr_route_ex; sequences of --seq-len rows)")
     ap.add_argument("--seq-len", type=int, default=0)
+    ap.add_argument("--fp8", action="store_true",
+                    help="decode workloads (n <= 64) on an 8-bit copy of W (tlr_create_fp8); the roofline then "
+                         "counts one byte per weight")
     ap.add_argument("--mlp", type=int, default=0,
                     help="attach a learned router of this hidden width (random weights) and route on its score")
     args = ap.parse_args()
