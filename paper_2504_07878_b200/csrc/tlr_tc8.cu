@@ -35,7 +35,10 @@ namespace tlr {
 
 namespace {
 
-constexpr int kBlockM = 128;                 // TMEM lanes; the MMA's M
+constexpr int kBlockM = 64;                  // the MMA's M: the kernel serves at most 64 token rows, and an M = 64
+                                             // instruction takes about two thirds of the time of an M = 128 one.
+                                             // Its accumulator row r lives in TMEM lane 32 * (r / 16) + r % 16:
+                                             // lanes 0..15 of each 32-lane quadrant (checked on the device).
 constexpr int kBlockN = 256;                 // max vocabulary rows per tile == accumulator columns
 constexpr int kSlabK = 128;                  // fp8 elements per slab row = 128 B = one swizzle span
 constexpr int kUmmaK8 = 32;                  // K of one kind::f8f6f4 MMA
@@ -48,7 +51,7 @@ constexpr int kMaxAStages = 8;
 constexpr int kMaxBStages = 8;
 constexpr int kRelease = 16;
 constexpr int kBarrierBytes = 512;
-constexpr int kScratchBytes = kBlockM * 16;
+constexpr int kScratchBytes = kBlockM * 16;   // one Partial per token row
 constexpr int kScaleBytes = kEpiWarps * kBlockN * 4;   // a tile's weight scales, one copy per epilogue warp
 constexpr int kSmemLimit = 232448;
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
@@ -332,14 +335,15 @@ tc8_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     const int grp = warp >= 7 ? 1 : 0;
     const int ewarp = grp * 4 + (warp & 3);
     const int quad = warp & 3;
-    const int row = quad * 32 + lane;
+    const int row = quad * 16 + (lane & 15);     // lanes 0..15 of the quadrant hold rows 16 quad .. 16 quad + 15
+    const bool has_row = lane < 16 && row < p.n; // lanes 16..31 of a quadrant hold nothing with M = 64
     float* ws = scale_area + ewarp * kBlockN;
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
     uint32_t ord = 0;
-    const bool warp_has_rows = quad * 32 < p.n;
-    const float hs = row < p.n ? p.hscale[row] : 1.0f;
+    const bool warp_has_rows = quad * 16 < p.n;
+    const float hs = has_row ? p.hscale[row] : 1.0f;
     for (int unit = worker; unit < units && ok; unit += workers, ++ord) {
       float m = -INFINITY, S = 0.f, cS = 0.f, Tq = 0.f, cT = 0.f;
       int idx = kNoToken;
@@ -442,7 +446,7 @@ tc8_projection_kernel(const __grid_constant__ CUtensorMap map_h,
       if (grp == 1) {
         if (ok && ord > 0) ok = mbar_wait(xch_empty(quad), (ord - 1) & 1u, abort_flag, p.status, wait_ns);
         if (ok) {
-          scratch[row] = out;
+          if (lane < 16) scratch[row] = out;
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_full(quad));
         }
@@ -453,7 +457,7 @@ tc8_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_empty(quad));
           out = merge(out, other);
-          if (row < p.n) p.partials[static_cast<size_t>(row) * p.chunks + chunk] = out;
+          if (has_row) p.partials[static_cast<size_t>(row) * p.chunks + chunk] = out;
         }
       }
     }
