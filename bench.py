@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc.cu", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
-    "sha256": "f59fe13215d784aaaf9774ee28ea5f9e26f10523198f646fd29ff2e415568a33",
-    "bytes_per_launch": {"decode256": 276.86e6, "decode16": 276.26e6, "sweep512": 531.56e6},
+    "sha256": "72a786f107dbdfbb2b4140ad0e09cbd4764eb5f3ff3746d89b0e268d84bfd847",
+    "bytes_per_launch": {"decode256": 276.50e6, "decode16": 277.03e6, "sweep512": 531.47e6},
 }
 
 

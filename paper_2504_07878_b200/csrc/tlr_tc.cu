@@ -187,6 +187,11 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
   if (warp != 0) asm volatile("griddepcontrol.wait;" ::: "memory");
   asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
+  // With at most 64 token rows (one CTA per worker) the MMAs run with M = 64: such an instruction takes
+  // about two thirds of the time of an M = 128 one, and the padding rows were wasted work anyway.  Its
+  // accumulator row r lives in TMEM lane 32 * (r / 16) + r % 16, i.e. in lanes 0..15 of each 32-lane
+  // quadrant (checked on the device), so an epilogue warp then holds 16 rows instead of 32.
+  const bool m64 = kCta == 1 && p.a_rows <= 64;
   const int k_slabs = (p.d + kBlockK - 1) / kBlockK;
   const int units = p.chunks * p.row_units;
   const int T = p.tiles_per_unit;
@@ -276,7 +281,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
         for (int t = 0; t < T && ok; ++t) {
           const Tile tl = tile_of<kCta>(p, unit, t, 0);
           if (tl.rows == 0) continue;
-          const uint32_t idesc = instr_desc(kBlockM * kCta, tl.rows);
+          const uint32_t idesc = instr_desc(m64 ? 64 : kBlockM * kCta, tl.rows);
           ok = __all_sync(0xffffffffu, mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status, wait_ns));
           if (!ok) break;
           tc_fence_after();
@@ -317,14 +322,15 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
     // ------------------------------------------------------------------ epilogue (warps 2-5, 7-10)
     const int grp = warp >= 7 ? 1 : 0;       // 0: lower half of a tile's columns, 1: upper half
     const int quad = warp & 3;               // TMEM lane quadrant this warp may read
-    const int row_in_cta = quad * 32 + lane;
+    const int row_in_cta = m64 ? quad * 16 + (lane & 15) : quad * 32 + lane;
+    const bool lane_has_row = !m64 || lane < 16;   // with M = 64 the upper half of a quadrant holds nothing
     int acc = 0;
     uint32_t acc_phase = 0;
     bool ok = true;
     uint32_t ord = 0;                        // ordinal of the unit among this worker's units
     for (int unit = worker; unit < units && ok; unit += workers, ++ord) {
       const Tile first = tile_of<kCta>(p, unit, 0, cta_rank);
-      const bool warp_has_rows = (first.row0 + quad * 32) < p.n;   // warp-uniform
+      const bool warp_has_rows = (first.row0 + (m64 ? quad * 16 : quad * 32)) < p.n;   // warp-uniform
       // Running summary of this thread's row over the unit.  S = sum 2^y and T = sum 2^y * y
       // with y = (z - m) * log2(e) <= 0; both are accumulated per 32-column group first and
       // then added with a compensated (Kahan) sum, so that one dominant term -- a confident
@@ -419,7 +425,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
       if (grp == 1) {
         if (ok && ord > 0) ok = mbar_wait(xch_empty(quad), (ord - 1) & 1u, abort_flag, p.status, wait_ns);
         if (ok) {
-          scratch[row_in_cta] = out;
+          if (lane_has_row) scratch[row_in_cta] = out;
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_full(quad));
         }
@@ -430,7 +436,7 @@ tc_projection_kernel(const __grid_constant__ CUtensorMap map_h,
           __syncwarp();
           if (lane == 0) mbar_arrive(xch_empty(quad));
           out = merge(out, other);
-          if (first.row0 + row_in_cta < p.n)
+          if (lane_has_row && first.row0 + row_in_cta < p.n)
             p.partials[static_cast<size_t>(first.row0 + row_in_cta) * p.chunks + first.chunk] = out;
         }
       }
