@@ -36,7 +36,7 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc.cu", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
-    "sha256": "72a786f107dbdfbb2b4140ad0e09cbd4764eb5f3ff3746d89b0e268d84bfd847",
+    "sha256": "06b0e7d9ace1da2464fade6a9fd2409357daa8602a903792937deb9dfb3c54ac",
     "bytes_per_launch": {"decode256": 276.50e6, "decode16": 277.03e6, "sweep512": 531.47e6},
 }
 

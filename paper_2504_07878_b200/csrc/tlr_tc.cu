@@ -4,7 +4,7 @@
 // the epilogue, so the n x V logits never leave the SM.
 //
 // Two instantiations of one kernel:
-//   kCta = 1  one CTA per worker, MMA M = 128 token rows            (n <= 128)
+//   kCta = 1  one CTA per worker, MMA M = 128 token rows            (n <= 128; M = 64 when n <= 64)
 //   kCta = 2  a cluster of two CTAs per worker, MMA M = 256 rows (cta_group::2): each
 //             CTA stages its own 128 rows of h and HALF of the W tile, and the pair's
 //             tensor cores read both halves, so a W byte enters shared memory once
