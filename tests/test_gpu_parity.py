@@ -24,6 +24,7 @@ PATHS = [pytest.param(1, id="simt"), pytest.param(2, id="tc")]
 SMALL_SHAPES = [
     (1, 64, 300), (16, 64, 1000), (37, 128, 4099), (130, 72, 5000), (257, 896, 3001),
     (300, 200, 20011), (129, 1536, 2500), (64, 2048, 777), (513, 64, 70000),
+    (64, 128, 3000), (65, 128, 3000), (49, 264, 1111),      # either side of the 64-row switch of the MMA's M
 ]
 
 
