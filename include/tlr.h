@@ -108,6 +108,9 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
  * Enqueues its kernels on cuda_stream and returns without synchronising; outputs are
  * valid once the stream reaches that point.  Allocates nothing.  Calls on one context
  * share its workspace, so they must be ordered (same stream, or externally serialised).
+ * Because it neither allocates, nor reads anything back, nor synchronises, the call may be
+ * captured in a CUDA graph (stream capture) and replayed: the graph then reads h and writes
+ * the outputs at the captured addresses, with the captured n and tau.
  * Errors (all detected on the host before any launch): TLR_ERR_ARG, TLR_ERR_ALIGN,
  * TLR_ERR_TOO_MANY_ROWS, TLR_ERR_CUDA.
  */
