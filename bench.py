@@ -285,8 +285,15 @@ def run_ours(args):
         roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s"}
     else:
         achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
-        peak = float(peaks.get("bf16_tflops_sustained" if ms_total > 1000 else "bf16_tflops", peaks["bf16_tflops"]))
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s"}
+        # Which measured cuBLAS figure the kernel is held against: the kernel-timing pass runs back to back
+        # right after the timed region, so by its end the GPU has been under continuous load for load_s
+        # seconds.  From one second on that is the power-capped regime of the "sustained" figure (the
+        # clocks in this line show it); a shorter run is compared with the burst figure.
+        load_s = (ms_total + kernel_ms * launches) * 1e-3
+        sustained = load_s >= 1.0
+        peak = float(peaks.get("bf16_tflops_sustained" if sustained else "bf16_tflops", peaks["bf16_tflops"]))
+        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
+                "peak_kind": "sustained" if sustained else "burst", "continuous_load_s": load_s}
     roof.update({"frac": achieved / peak, "traffic": None if fp8 else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
                  "peak_source": "of " + peak_kind,
                  "kernel": ("h_split_kernel + tc8_projection_kernel" if fp8 else
@@ -294,6 +301,8 @@ def run_ours(args):
                  "kernel_ms": kernel_ms, "kernel_launches_timed": launches,
                  "tensor_frac_same_launch": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
                  float(peaks["bf16_tflops"]),
+                 "tensor_frac_of_sustained": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
+                 float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
                  "hbm_frac_same_launch": algorithmic_bytes(n, d, V, fp8) / (kernel_ms * 1e-3) / 1e9 /
                  float(peaks["hbm_gbs"])})
 
