@@ -153,14 +153,14 @@ void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
   if (c->fp8) {
     tlr::Tc8Config cfg;
     tlr::TcPlan tp;
-    tlr::tc8_configure(n, &cfg);
+    tlr::tc8_configure(n, c->d, &cfg);
     tlr::tc_plan(n <= 128 ? n : 128, c->V, 1, c->sm_count, tlr::kMaxChunks, &tp);
     out->vocab_chunks = tp.chunks;
     out->row_units = 1;
     out->grid = tp.chunks < c->sm_count ? tp.chunks : c->sm_count;
     out->block = tlr::tc8_threads();
     out->smem_bytes = cfg.smem_bytes;
-    out->launches = n > 0 ? 3 : 1;
+    out->launches = n > 0 ? (cfg.inline_split ? 2 : 3) : 1;
   } else if (path == TLR_PATH_TC) {
     tlr::TcConfig cfg;
     tlr::TcPlan tp;
@@ -217,9 +217,10 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
   if (ctx->fp8) {
     tlr::Tc8Config cfg;
     tlr::TcPlan tp;
-    tlr::tc8_configure(n, &cfg);
+    tlr::tc8_configure(n, ctx->d, &cfg);
     tlr::tc_plan(n, ctx->V, 1, ctx->sm_count, tlr::kMaxChunks, &tp);
-    if (tlr::launch_h_split(h_bf16_dev, n, ctx->d, cfg.a_rows, ctx->h_parts, ctx->hscale, stream) != cudaSuccess)
+    if (!cfg.inline_split &&
+        tlr::launch_h_split(h_bf16_dev, n, ctx->d, cfg.a_rows, ctx->h_parts, ctx->hscale, stream) != cudaSuccess)
       return TLR_ERR_CUDA;
     CUtensorMap map_h;
     if (!make_map8(ctx, &map_h, ctx->h_parts, 2 * cfg.a_rows, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
@@ -236,6 +237,8 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
     p.b_stages = cfg.b_stages;
     p.wait_limit_ns = ctx->debug_wait_ns;
     p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
+    p.inline_split = cfg.inline_split;
+    p.h = h_bf16_dev;
     p.hscale = ctx->hscale;
     p.wscale = ctx->wscale;
     p.partials = ctx->partials;

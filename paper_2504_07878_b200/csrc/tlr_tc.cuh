@@ -41,6 +41,8 @@ struct Tc8Config {
   int a_rows;       // rows of an h slab part held in shared memory (16..64)
   int a_stages;     // depth of the h ring (a stage = both parts of one 128-wide slab)
   int b_stages;     // depth of the W ring (a stage = up to 256 rows x 128 bytes)
+  int inline_split; // 1: n <= 16 and the two parts of all of h fit in shared memory -- the kernel splits h itself
+                    // at its start and keeps it resident (a_stages == number of K slabs); no split kernel runs
   int smem_bytes;
 };
 
@@ -50,6 +52,8 @@ struct Tc8Params {
   int a_rows, a_stages, b_stages;
   unsigned long long wait_limit_ns;
   int debug_drop_w_copies;
+  int inline_split;
+  const void* h;         // bf16 [n][d], read when inline_split
   const float* hscale;   // [n] power-of-two scale of every row of h (written by the split kernel)
   const float* wscale;   // [V] scale of every row of W
   Partial* partials;     // [n][chunks]
@@ -58,7 +62,7 @@ struct Tc8Params {
 
 int tc8_threads();
 int tc8_max_rows();
-void tc8_configure(int n, Tc8Config* c);
+void tc8_configure(int n, int d, Tc8Config* c);
 cudaError_t tc8_prepare();
 // h [n][d] bf16 -> parts [2][rows_alloc][d] e4m3 (rows n.. zero) and hscale[n]
 cudaError_t launch_h_split(const void* h_bf16, int n, int d, int rows_alloc, uint8_t* parts, float* hscale,

@@ -55,7 +55,8 @@ def test_fp8_head_matches_oracle_on_dequantised_matrix(pkg, n, d, V):
     tau = O.percentile_tau(first.conf, 0.5) if n > 1 else 0.5
     ref = O.route_oracle(S.bf16_bits(h), None, tau, W64=W64)
     gpu = run_fp8(pkg, codes, scale, h, tau)
-    assert gpu["status"] == 0 and gpu["plan"].launches == 3
+    assert gpu["status"] == 0
+    assert gpu["plan"].launches == (2 if n <= 16 and d <= 1024 else 3)   # small batches of a small head: the kernel splits h itself
     check_self_consistency(gpu, tau, V)
     rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(h)), W64)
     if rep["route_exempt_rows"] == 0:
