@@ -199,6 +199,55 @@ void free_all(tlr_ctx* c) {
   delete c;
 }
 
+// What both kinds of context share: the device check, the workspace, the staging buffers of
+// tlr_route_host and the driver's tensor-map encoder (c->encode stays null if it cannot be had).
+tlr_status new_context(int d, int V, const void* W_dev, int max_n, tlr_ctx** out) {
+  if (static_cast<long long>(V) + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return TLR_ERR_CUDA;
+  cudaDeviceProp prop;
+  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TLR_ERR_CUDA;
+  if (prop.major != 10) return TLR_ERR_UNSUPPORTED;   // the kernels are built for sm_100a only
+  tlr_ctx* c = new (std::nothrow) tlr_ctx();
+  if (c == nullptr) return TLR_ERR_NOMEM;
+  c->device = dev;
+  c->sm_count = prop.multiProcessorCount;
+  c->d = d;
+  c->V = V;
+  c->max_n = max_n;
+  c->W = W_dev;
+  const size_t np = static_cast<size_t>(max_n);
+  bool ok = true;
+  ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
+  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
+  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
+  if (!ok) {
+    cudaGetLastError();
+    free_all(c);
+    return TLR_ERR_NOMEM;
+  }
+  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
+    cudaGetLastError();
+    c->out_mapped = nullptr;   // tlr_route_host then stages the outputs in device memory and copies them
+  }
+  if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
+      cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
+    free_all(c);
+    return TLR_ERR_CUDA;
+  }
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+      qres == cudaDriverEntryPointSuccess && fn != nullptr)
+    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
+  cudaGetLastError();
+  *out = c;
+  return TLR_OK;
+}
+
 // Enqueues the projection kernel of a call with n > 0 rows: chunk partials into ctx->partials.
 tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const tlr_plan& plan, cudaStream_t stream) {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
@@ -316,59 +365,16 @@ tlr_status tlr_create(int32_t d, int32_t V, const void* W_bf16_dev, int32_t max_
   *out = nullptr;
   if (d <= 0 || V <= 0 || max_n <= 0 || W_bf16_dev == nullptr) return TLR_ERR_ARG;
   if ((reinterpret_cast<uintptr_t>(W_bf16_dev) & 15u) != 0) return TLR_ERR_ALIGN;
-  if (static_cast<long long>(V) + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
-
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return TLR_ERR_CUDA;
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TLR_ERR_CUDA;
-  if (prop.major != 10) return TLR_ERR_UNSUPPORTED;   // the kernels are built for sm_100a only
-
-  tlr_ctx* c = new (std::nothrow) tlr_ctx();
-  if (c == nullptr) return TLR_ERR_NOMEM;
-  c->device = dev;
-  c->sm_count = prop.multiProcessorCount;
-  c->d = d;
-  c->V = V;
-  c->max_n = max_n;
-  c->W = W_bf16_dev;
-
-  const size_t np = static_cast<size_t>(max_n);
-  bool ok = true;
-  ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
-  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
-  if (!ok) {
-    cudaGetLastError();
-    free_all(c);
-    return TLR_ERR_NOMEM;
-  }
-  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
-    cudaGetLastError();
-    c->out_mapped = nullptr;   // tlr_route_host then stages the outputs in device memory and copies them
-  }
-  if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
-      cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
-    free_all(c);
-    return TLR_ERR_CUDA;
-  }
+  tlr_ctx* c = nullptr;
+  const tlr_status st = new_context(d, V, W_bf16_dev, max_n, &c);
+  if (st != TLR_OK) return st;
 
   // Tensor-core path: needs 16-byte row pitch for TMA, and the driver's tensor-map encoder.
-  c->tc_ok = false;
   if (d % 8 == 0) {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qres;
-    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
-        qres == cudaDriverEntryPointSuccess && fn != nullptr) {
-      c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-      if (make_map(c, &c->map_w128, W_bf16_dev, V, d, 128) && make_map(c, &c->map_w64, W_bf16_dev, V, d, 64) && make_map(c, &c->map_w16, W_bf16_dev, V, d, 16) &&
-          tlr::tc_prepare() == cudaSuccess) {
-        c->tc_ok = true;
-      }
-    }
+    if (c->encode != nullptr && make_map(c, &c->map_w128, W_bf16_dev, V, d, 128) &&
+        make_map(c, &c->map_w64, W_bf16_dev, V, d, 64) && make_map(c, &c->map_w16, W_bf16_dev, V, d, 16) &&
+        tlr::tc_prepare() == cudaSuccess)
+      c->tc_ok = true;
     cudaGetLastError();
     if (!c->tc_ok) {   // on an sm_100 device with d % 8 == 0 this must work; do not fall back silently
       free_all(c);
@@ -387,56 +393,21 @@ tlr_status tlr_create_fp8(int32_t d, int32_t V, const void* W_e4m3_dev, const fl
   if ((reinterpret_cast<uintptr_t>(W_e4m3_dev) & 15u) != 0 || (reinterpret_cast<uintptr_t>(wscale_dev) & 3u) != 0)
     return TLR_ERR_ALIGN;
   if (d % 16 != 0) return TLR_ERR_UNSUPPORTED;         // rows of 8-bit W must be multiples of 16 bytes for TMA
-  if (static_cast<long long>(V) + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess) return TLR_ERR_CUDA;
-  cudaDeviceProp prop;
-  if (cudaGetDeviceProperties(&prop, dev) != cudaSuccess) return TLR_ERR_CUDA;
-  if (prop.major != 10) return TLR_ERR_UNSUPPORTED;
-  tlr_ctx* c = new (std::nothrow) tlr_ctx();
-  if (c == nullptr) return TLR_ERR_NOMEM;
-  c->device = dev;
-  c->sm_count = prop.multiProcessorCount;
-  c->d = d;
-  c->V = V;
-  c->max_n = max_n;
-  c->W = W_e4m3_dev;
+  tlr_ctx* c = nullptr;
+  const tlr_status st = new_context(d, V, W_e4m3_dev, max_n, &c);
+  if (st != TLR_OK) return st;
   c->wscale = wscale_dev;
   c->fp8 = true;
-  const size_t np = static_cast<size_t>(max_n);
   const size_t rows8 = static_cast<size_t>(tlr::tc8_max_rows());
-  bool ok = true;
-  ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
-  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->h_parts, 2 * rows8 * d) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->hscale, rows8 * sizeof(float)) == cudaSuccess;
-  if (!ok) {
+  if (cudaMalloc(&c->h_parts, 2 * rows8 * d) != cudaSuccess || cudaMalloc(&c->hscale, rows8 * sizeof(float)) != cudaSuccess) {
     cudaGetLastError();
     free_all(c);
     return TLR_ERR_NOMEM;
   }
-  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
-    cudaGetLastError();
-    c->out_mapped = nullptr;
-  }
-  if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
-      cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
-    free_all(c);
-    return TLR_ERR_CUDA;
-  }
-  void* fn = nullptr;
-  cudaDriverEntryPointQueryResult qres;
-  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
-      qres == cudaDriverEntryPointSuccess && fn != nullptr) {
-    c->encode = reinterpret_cast<EncodeTiledFn>(fn);
-    if (make_map8(c, &c->map_w128, W_e4m3_dev, V, d, 128) && make_map8(c, &c->map_w64, W_e4m3_dev, V, d, 64) &&
-        make_map8(c, &c->map_w16, W_e4m3_dev, V, d, 16) && tlr::tc8_prepare() == cudaSuccess)
-      c->tc_ok = true;
-  }
+  if (c->encode != nullptr && make_map8(c, &c->map_w128, W_e4m3_dev, V, d, 128) &&
+      make_map8(c, &c->map_w64, W_e4m3_dev, V, d, 64) && make_map8(c, &c->map_w16, W_e4m3_dev, V, d, 16) &&
+      tlr::tc8_prepare() == cudaSuccess)
+    c->tc_ok = true;
   cudaGetLastError();
   if (!c->tc_ok) {
     free_all(c);
