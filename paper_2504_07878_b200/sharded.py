@@ -38,18 +38,25 @@ def gather_summaries(local: torch.Tensor, group=None) -> torch.Tensor:
 class VocabShardedRouter:
     """Owner of one rank's context (on its rows of W), its summary buffers and the output tensors."""
 
-    def __init__(self, W_shard: torch.Tensor, v_offset: int, max_n: int, world: int, group=None):
-        if not (W_shard.is_cuda and W_shard.dtype == torch.bfloat16 and W_shard.dim() == 2
-                and W_shard.is_contiguous()):
-            raise ValueError("W_shard must be a contiguous CUDA bf16 [V_local, d] tensor")
+    def __init__(self, W_shard: torch.Tensor, v_offset: int, max_n: int, world: int, group=None, wscale=None):
+        """W_shard: this rank's rows of W, bf16 [V_local, d]; or, with wscale (float32 [V_local]), their e4m3 codes
+        (decode batches of up to 64 rows, see tlr_create_fp8)."""
+        fp8 = wscale is not None
+        ok_dtype = W_shard.dtype in (torch.uint8, torch.float8_e4m3fn) if fp8 else W_shard.dtype == torch.bfloat16
+        if not (W_shard.is_cuda and ok_dtype and W_shard.dim() == 2 and W_shard.is_contiguous()):
+            raise ValueError("W_shard must be a contiguous CUDA [V_local, d] tensor, bf16 or (with wscale) e4m3 codes")
         self.W = W_shard
+        self.wscale = wscale
         self.v_offset = int(v_offset)
         self.world = int(world)
         self.group = group
         self.max_n = max_n
         dev = W_shard.device
         with torch.cuda.device(dev):
-            self.ctx = B.tlr_create(W_shard.shape[1], W_shard.shape[0], W_shard, max_n)
+            if fp8:
+                self.ctx = B.tlr_create_fp8(W_shard.shape[1], W_shard.shape[0], W_shard, wscale, max_n)
+            else:
+                self.ctx = B.tlr_create(W_shard.shape[1], W_shard.shape[0], W_shard, max_n)
             self.summary = torch.empty((max_n, 4), dtype=torch.float32, device=dev)     # 16 bytes per row
             self.token = torch.empty(max_n, dtype=torch.int32, device=dev)
             self.conf = torch.empty(max_n, dtype=torch.float32, device=dev)

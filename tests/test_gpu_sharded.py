@@ -102,3 +102,31 @@ def test_shard_argument_errors(pkg):
         pkg.tlr_shard_finish(r.ctx, r.summary, 0, 4, 0.5, r.token, r.conf, r.entropy, r.route_mask, r.routed_idx,
                              r.routed_count)                 # zero shards
     r.close()
+
+
+def test_sharded_8bit_head(pkg):
+    """Shards of an e4m3 head (codes and scales cut at the same rows), merged, against the oracle on the
+    de-quantised matrix."""
+    n, d, V, shards = 24, 128, 5000, 3
+    codes, scale = S.make_W8(d, V, seed=8, std=0.1)
+    W64 = O.dequantize_e4m3(codes.numpy(), scale.numpy())
+    h = S.make_h(n, d, seed=8).h
+    ref = O.route_oracle(S.bf16_bits(h), None, 0.5, W64=W64)
+    cd, sd, hd = codes.cuda(), scale.cuda(), h.cuda()
+    routers, parts = [], []
+    for g in range(shards):
+        v0, v1 = pkg.shard_bounds(V, shards, g)
+        r = pkg.VocabShardedRouter(cd[v0:v1], v0, max_n=n, world=shards, wscale=sd[v0:v1])
+        parts.append(r.summarize(hd).clone())
+        routers.append(r)
+    last = routers[-1]
+    last.finish(torch.stack(parts).contiguous(), n, 0.5)
+    torch.cuda.synchronize()
+    gpu = {"token": to_np(last.token[:n]), "conf": to_np(last.conf[:n]), "entropy": to_np(last.entropy[:n]),
+           "route_mask": to_np(last.route_mask[:n]), "routed_idx": to_np(last.routed_idx),
+           "routed_count": int(last.routed_count.item())}
+    check_self_consistency(gpu, 0.5, V)
+    check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(h)), W64)
+    for r in routers:
+        assert pkg.tlr_last_device_status(r.ctx) == 0
+        r.close()
