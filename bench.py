@@ -35,7 +35,7 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # captures summarised under profiles/.  Only valid for the kernel source they were taken on: the
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
-    "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc.cu", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
+    "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc_kernel.cuh", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
     "sha256": "06b0e7d9ace1da2464fade6a9fd2409357daa8602a903792937deb9dfb3c54ac",
     "bytes_per_launch": {"decode256": 276.50e6, "decode16": 277.03e6, "sweep512": 531.47e6},
 }
@@ -137,6 +137,90 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
+def roofline_fractions(n, d, V, seconds, peaks, fp8=False):
+    """The three fractions every record carries, from one duration: HBM, tensor against the burst cuBLAS
+    figure, tensor against the sustained one; and the ridge reading max(t_mem, t_mma) / t with t_mma at the
+    burst figure (both pipes would be busy for the longer of the two times at best)."""
+    by, fl = algorithmic_bytes(n, d, V, fp8), algorithmic_flops(n, d, V)
+    t_mem = by / (float(peaks["hbm_gbs"]) * 1e9)
+    t_mma = fl / (float(peaks["bf16_tflops"]) * 1e12)
+    t_mma_sus = fl / (float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * 1e12)
+    return {"hbm_frac": t_mem / seconds, "tensor_frac_burst": t_mma / seconds,
+            "tensor_frac_sustained": t_mma_sus / seconds, "ridge_frac": max(t_mem, t_mma) / seconds}
+
+
+def time_steps(P, routers, step, steps, sampler, world, kernel_steps):
+    """K steps between two CUDA events on the launching stream (clocks sampled meanwhile), then, back to
+    back, `kernel_steps` more steps with the projection kernel bracketed by events inside tlr_route.
+    Returns (ms per step, ms per projection launch, projection launches timed, seconds of continuous load)."""
+    stream = torch.cuda.current_stream()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    while not e1.query():
+        sampler.sample()
+        time.sleep(0.002)
+    sampler.sample()
+    for r in routers:
+        P.tlr_set_kernel_timing(r.ctx, True)
+    for i in range(kernel_steps):
+        step(i)
+    e2 = torch.cuda.Event(enable_timing=True)
+    e2.record(stream)
+    while not e2.query():
+        sampler.sample()
+        time.sleep(0.002)
+    torch.cuda.synchronize()
+    ms_total = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
+    load_s = e0.elapsed_time(e2) * 1e-3
+    launches, kms = 0, 0.0
+    for r in routers:
+        ln, ms = P.tlr_read_kernel_timing(r.ctx)
+        launches += ln
+        kms += ms
+        P.tlr_set_kernel_timing(r.ctx, False)
+    return ms_total / steps, kms / max(launches, 1), launches, load_s
+
+
+def side_record(P, name, routers, h_dev, tau, seconds, gpu_index, peaks, fp8=False):
+    """One more workload on heads that are already resident: about `seconds` of back-to-back steps."""
+    wl = S.WORKLOADS[name]
+    n, d, V = wl.n, wl.d, wl.V
+    stream = torch.cuda.current_stream()
+
+    def step(i):
+        routers[i % len(routers)].route(h_dev, tau, stream)
+
+    for i in range(5):
+        step(i)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(4):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    per = max(e0.elapsed_time(e1) / 4 * 1e-3, 1e-6)
+    steps = int(max(20, min(20000, seconds / per)))
+    ksteps = int(max(10, min(steps // 2, 4000)))
+    sampler = ClockSampler(gpu_index)
+    ms, kms, launches, load_s = time_steps(P, routers, step, steps, sampler, 1, ksteps)
+    status = max(P.tlr_last_device_status(r.ctx) for r in routers)
+    if status & P.TLR_DEV_WAIT_TIMEOUT:
+        raise SystemExit("device status flags raised in the %s record: %d" % (name, status))
+    rec = {"workload": "%s%s: n=%d rows, d=%d, V=%d, tau=%g" % (name, " with an 8-bit copy of W" if fp8 else "", n, d, V, tau),
+           "steps": steps, "ms_per_step": ms, "value": n / (ms * 1e-3), "unit": UNIT,
+           "kernel_ms": kms, "kernel_launches_timed": launches, "continuous_load_s": load_s,
+           "bound": "hbm" if n <= RIDGE_ROWS_HBM else "tensor", "clocks": sampler.summary(),
+           "routed_rows_per_step": int(routers[0].routed_count.item())}
+    rec["kernel"] = roofline_fractions(n, d, V, kms * 1e-3, peaks, fp8)
+    rec["step"] = roofline_fractions(n, d, V, ms * 1e-3, peaks, fp8)
+    rec["frac"] = rec["kernel"]["hbm_frac" if n <= RIDGE_ROWS_HBM else "tensor_frac_burst"]
+    return rec
+
+
 def run_ours(args):
     import paper_2504_07878_b200 as P
     from paper_2504_07878_b200 import build
@@ -158,6 +242,8 @@ def run_ours(args):
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
         dist.barrier()
     P.load_library()
+    gpu_index = physical_gpu_index(local_rank)
+    peaks, peak_kind = measured_peaks()
 
     wl = S.WORKLOADS[args.workload]
     n, d, V = wl.n, wl.d, wl.V
@@ -215,38 +301,16 @@ def run_ours(args):
         step(i)
     barrier()
 
-    # ---- timed region: exactly K steps, device time between two events, clocks sampled meanwhile
-    sampler = ClockSampler(physical_gpu_index(local_rank))
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record(stream)
-    for i in range(args.steps):
-        step(i)
-    e1.record(stream)
-    while not e1.query():
-        sampler.sample()
-        time.sleep(0.002)
-    sampler.sample()
+    # ---- timed region: exactly K steps, device time between two events, clocks sampled meanwhile;
+    # then, back to back, the dominant kernel alone (bracketed by events inside tlr_route)
+    sampler = ClockSampler(gpu_index)
+    ms_per_step, kernel_ms, launches, load_s = time_steps(P, routers, step, args.steps, sampler, world,
+                                                          min(args.steps, 2000))
     barrier()
-    ms_total = max_over_ranks(e0.elapsed_time(e1), world, "cuda")
     status = max(P.tlr_last_device_status(r.ctx) for r in routers)
     if status & P.TLR_DEV_WAIT_TIMEOUT:
         raise SystemExit("device status flags raised during the timed region: %d" % status)
     routed = int(routers[0].routed_count.item())
-
-    # ---- dominant kernel alone: the projection kernel bracketed by events inside tlr_route
-    for r in routers:
-        P.tlr_set_kernel_timing(r.ctx, True)
-    ksteps = min(args.steps, 2000)
-    for i in range(ksteps):
-        step(i)
-    torch.cuda.synchronize()
-    launches, kms = 0, 0.0
-    for r in routers:
-        ln, ms = P.tlr_read_kernel_timing(r.ctx)
-        launches += ln
-        kms += ms
-        P.tlr_set_kernel_timing(r.ctx, False)
-    kernel_ms = kms / max(launches, 1)
 
     # ---- end to end through the host-buffer entry point (pinned host memory)
     h_pin = hid.h.pin_memory()
@@ -269,42 +333,73 @@ def run_ours(args):
         host_step(i)
     torch.cuda.synchronize()
     e2e_s = max_over_ranks(time.perf_counter() - t0, world, "cuda")
-    e2e_routed = int(o_cnt.item())
     h2d = n * d * 2
     d2h = 17 * n + 4 + 4      # the six outputs in one block (routed_idx at full capacity) + the status word
 
+    # ---- the same step under sustained load, and the other regimes of the target on the same head
+    sustained = None
+    also = []
+    if world == 1 and args.extras and args.workload == "decode256" and not fp8 and not variant_args:
+        sustained = side_record(P, "decode256", routers, h_dev, tau, 1.5, gpu_index, peaks)
+        sustained["note"] = ("the benchmark step back to back for about 1.5 s, then the kernel-timing pass: the "
+                             "power-capped regime; compare time x clocks.sm_mhz with the short run above")
+        torch.cuda.synchronize()
+        time.sleep(0.5)
+        wl16 = S.WORKLOADS["decode16"]
+        r16 = [P.Router(w, max_n=wl16.n) for w in Ws]
+        also.append(side_record(P, "decode16", r16, S.make_h(wl16.n, d, seed=0).h.cuda(), 0.5, 0.3, gpu_index, peaks))
+        for r in r16:
+            r.close()
+        wlp = S.WORKLOADS["prefill8192"]
+        rp = [P.Router(w, max_n=wlp.n) for w in Ws]
+        hp = S.make_h(wlp.n, d, seed=0, W=W_host, planted_fraction=wlp.planted_fraction).h.cuda()
+        also.append(side_record(P, "prefill8192", rp, hp, wlp.tau, 1.2, gpu_index, peaks))
+        for r in rp:
+            r.close()
+        del rp, hp
+        codes, wscale = S.make_W8(d, V, seed=0)
+        W8 = [(codes.cuda(), wscale.cuda()) for _ in range(copies)]
+        r8 = [P.Router(c, max_n=wl16.n, wscale=sc) for c, sc in W8]
+        also.append(side_record(P, "decode16", r8, S.make_h(wl16.n, d, seed=0).h.cuda(), 0.5, 0.3, gpu_index, peaks,
+                                fp8=True))
+        for r in r8:
+            r.close()
+        del r8, W8
+
+    # ---- N > 1: the vocabulary-sharded form of the same decode batch (one exchange step per call)
+    vocab_sharded = None
+    if world > 1 and n <= 1024 and not fp8 and not variant_args:
+        vocab_sharded = vocab_sharded_record(P, W_host, S.make_h(n, d, seed=0).h, tau, rank, world, args.steps,
+                                             max(args.warmup, 3))
+
     if rank != 0:
         return
-    peaks, peak_kind = measured_peaks()
-    ms_per_step = ms_total / args.steps
     value = job_throughput(world, n, ms_per_step * 1e-3)
+    kfr = roofline_fractions(n, d, V, kernel_ms * 1e-3, peaks, fp8)
+    sfr = roofline_fractions(n, d, V, ms_per_step * 1e-3, peaks, fp8)
     hbm_bound = n <= RIDGE_ROWS_HBM
     if hbm_bound:
         achieved = algorithmic_bytes(n, d, V, fp8) / (kernel_ms * 1e-3) / 1e9
-        peak = float(peaks["hbm_gbs"])
-        roof = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s"}
+        roof = {"bound": "hbm", "achieved": achieved, "peak": float(peaks["hbm_gbs"]), "unit": "GB/s",
+                "frac": kfr["hbm_frac"]}
     else:
+        # always held against the burst cuBLAS figure; the fraction of the sustained figure is beside it
         achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
-        # Which measured cuBLAS figure the kernel is held against: the kernel-timing pass runs back to back
-        # right after the timed region, so by its end the GPU has been under continuous load for load_s
-        # seconds.  From one second on that is the power-capped regime of the "sustained" figure (the
-        # clocks in this line show it); a shorter run is compared with the burst figure.
-        load_s = (ms_total + kernel_ms * launches) * 1e-3
-        sustained = load_s >= 1.0
-        peak = float(peaks.get("bf16_tflops_sustained" if sustained else "bf16_tflops", peaks["bf16_tflops"]))
-        roof = {"bound": "tensor", "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "peak_kind": "sustained" if sustained else "burst", "continuous_load_s": load_s}
-    roof.update({"frac": achieved / peak, "traffic": None if fp8 else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
-                 "peak_source": "of " + peak_kind,
+        roof = {"bound": "tensor", "achieved": achieved, "peak": float(peaks["bf16_tflops"]), "unit": "TFLOP/s",
+                "frac": kfr["tensor_frac_burst"], "peak_kind": "burst"}
+    roof.update({"traffic": None if fp8 else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
+                 "algorithmic_flops": algorithmic_flops(n, d, V), "peak_source": "of " + peak_kind,
                  "kernel": ("h_split_kernel + tc8_projection_kernel" if fp8 else
                             "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel"),
-                 "kernel_ms": kernel_ms, "kernel_launches_timed": launches,
-                 "tensor_frac_same_launch": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
-                 float(peaks["bf16_tflops"]),
-                 "tensor_frac_of_sustained": algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12 /
-                 float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])),
-                 "hbm_frac_same_launch": algorithmic_bytes(n, d, V, fp8) / (kernel_ms * 1e-3) / 1e9 /
-                 float(peaks["hbm_gbs"])})
+                 "kernel_ms": kernel_ms, "kernel_launches_timed": launches, "continuous_load_s": load_s,
+                 # the projection kernel alone (timed by events inside tlr_route, which also switch off the
+                 # overlap of its prologue with the previous merge kernel) and the whole step (projection +
+                 # merge launches, as timed for tokens/s), each against all three peaks and the ridge bound
+                 "kernel_fracs": kfr, "step_fracs": sfr,
+                 "step_frac": sfr["hbm_frac"] if hbm_bound else sfr["tensor_frac_burst"],
+                 "ridge_frac": kfr["ridge_frac"],
+                 "hbm_frac_same_launch": kfr["hbm_frac"], "tensor_frac_same_launch": kfr["tensor_frac_burst"],
+                 "tensor_frac_of_sustained": kfr["tensor_frac_sustained"]})
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
@@ -323,14 +418,55 @@ def run_ours(args):
                                 if "seq_len" in variant_args else "none") +
                                ("; learned router, hidden width %d" % args.mlp if args.mlp > 0 else "")},
         "e2e": {"value": job_throughput(world, n, e2e_s / esteps), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)"},
-        "gpu_launches": (int(plan.launches) + (1 if args.mlp > 0 else 0)) * args.steps,
+                "d2h_bytes_per_step": d2h, "steps": esteps, "api": "tlr_route_host (pinned host buffers)",
+                "frac_of_device_rate": (ms_per_step * 1e-3) / (e2e_s / esteps)},
+        # (a learned router runs inside the projection launch wherever the tensor-core kernel does: d % 8 == 0)
+        "gpu_launches": (int(plan.launches) + (1 if args.mlp > 0 and (fp8 or d % 8 != 0) else 0)) * args.steps,
         "clocks": sampler.summary(),
         "roofline": roof,
     }
+    if sustained is not None:
+        out["sustained"] = sustained
+    if also:
+        out["also"] = also
+    if vocab_sharded is not None:
+        out["vocab_sharded"] = vocab_sharded
     if world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, W_host, hid, tau, budget_s=15.0, w8=(codes, wscale) if fp8 else None)
     print(json.dumps(out))
+
+
+def vocab_sharded_record(P, W_host, h_cpu, tau, rank, world, steps, warmup):
+    """The same batch with the vocabulary sharded over the ranks (each holds V / world rows of W): projection
+    on the shard, one all-gather of n x 16 bytes per rank over NCCL, merge and decision on every rank.  Total
+    work is fixed as N grows (strong scaling of one decode batch); time is the max over ranks."""
+    import torch.distributed as dist
+    V = W_host.shape[0]
+    n = h_cpu.shape[0]
+    v0, v1 = P.shard_bounds(V, world, rank)
+    copies = 2          # two copies of the shard alternate, as in the main loop (a shard may fit in L2)
+    shards = [W_host[v0:v1].cuda() for _ in range(copies)]
+    rs = [P.VocabShardedRouter(w, v0, max_n=n, world=world) for w in shards]
+    h_dev = h_cpu.cuda()
+    stream = torch.cuda.current_stream()
+    for i in range(warmup):
+        rs[i % copies].route(h_dev, tau)
+    dist.barrier()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        rs[i % copies].route(h_dev, tau)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    dist.barrier()
+    ms = max_over_ranks(e0.elapsed_time(e1), world, "cuda") / steps
+    routed = int(rs[(steps - 1) % copies].routed_count.item())
+    for r in rs:
+        r.close()
+    return {"ms_per_step": ms, "value": n / (ms * 1e-3), "unit": UNIT, "scaling": "strong", "shards": world,
+            "rows_of_W_per_rank": v1 - v0, "routed_rows_per_step": routed,
+            "exchange": "NCCL all-gather of %d bytes per rank per step" % (16 * n)}
 
 
 def blas_threads():
@@ -413,6 +549,9 @@ def main():
     ap.add_argument("--workload", default="decode256", choices=sorted(S.WORKLOADS))
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extras", dest="extras", action="store_false",
+                    help="default workload only: skip the sustained-load record and the decode16 / prefill8192 / "
+                         "8-bit records that reuse the resident head")
     ap.add_argument("--tau", type=float, default=None, help="override the workload's threshold")
     ap.add_argument("--variants", action="store_true",
                     help="route with per-row thresholds and report the first routed position per sequence "

@@ -267,13 +267,16 @@ tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms);
 /*
  * tlr_debug_plan_tiles -- host-only view of the tensor-core kernel's static schedule for n rows,
  * a vocabulary of V and sm_count SMs (no GPU needed; used by the CPU tests of the planner).
+ * mlp_hidden > 0 plans the launch with a learned router of that hidden width inside it: the rows of
+ * its first layer are walked as one more unit per row unit and are reported as vocabulary rows
+ * V .. V + mlp_hidden (rounded up to the granule).
  * Writes up to `capacity` records of five int32 {worker, unit, first token row, first vocabulary
  * row, vocabulary rows} -- one per tile, in the order the workers walk them -- and the total
  * number of tiles to *count.  plan_out (optional) receives grid, chunks, row units and, in
  * `reserved`, the granule size in rows.
  */
-tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t* out, int32_t capacity,
-                                int32_t* count, tlr_plan* plan_out);
+tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t mlp_hidden, int32_t* out,
+                                int32_t capacity, int32_t* count, tlr_plan* plan_out);
 
 /* tlr_plan_query -- the launch plan a call with n rows would use.  No device work. */
 tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out);

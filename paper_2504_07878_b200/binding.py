@@ -59,7 +59,7 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_route.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_route_ex.argtypes = [P, P, c_int32, c_float, POINTER(TlrRouteOptions), P, P, P, P, P, P, P]
     lib.tlr_route_ex.restype = c_int32
-    lib.tlr_debug_plan_tiles.argtypes = [c_int32, c_int32, c_int32, P, c_int32, POINTER(c_int32), POINTER(TlrPlan)]
+    lib.tlr_debug_plan_tiles.argtypes = [c_int32, c_int32, c_int32, c_int32, P, c_int32, POINTER(c_int32), POINTER(TlrPlan)]
     lib.tlr_debug_plan_tiles.restype = c_int32
     lib.tlr_debug_inject.argtypes = [P, c_int32, c_uint32]
     lib.tlr_debug_inject.restype = c_int32
@@ -199,15 +199,17 @@ def tlr_debug_inject(ctx, kind: int, wait_limit_ms: int = 0):
     _check(load_library().tlr_debug_inject(ctx, kind, wait_limit_ms), "tlr_debug_inject")
 
 
-def tlr_debug_plan_tiles(n: int, V: int, sm_count: int = 148):
-    """Host-only: the tensor-core kernel's tile schedule as an int32 array [tiles, 5] and its plan."""
+def tlr_debug_plan_tiles(n: int, V: int, sm_count: int = 148, mlp_hidden: int = 0):
+    """Host-only: the tensor-core kernel's tile schedule as an int32 array [tiles, 5] and its plan
+    (mlp_hidden > 0: with a learned router of that width inside the launch)."""
     import numpy as np
     lib = load_library()
     count, plan = c_int32(0), TlrPlan()
-    _check(lib.tlr_debug_plan_tiles(n, V, sm_count, c_void_p(0), 0, byref(count), byref(plan)), "tlr_debug_plan_tiles")
-    out = np.zeros((count.value, 5), dtype=np.int32)
-    _check(lib.tlr_debug_plan_tiles(n, V, sm_count, c_void_p(out.ctypes.data), count.value, byref(count), byref(plan)),
+    _check(lib.tlr_debug_plan_tiles(n, V, sm_count, mlp_hidden, c_void_p(0), 0, byref(count), byref(plan)),
            "tlr_debug_plan_tiles")
+    out = np.zeros((count.value, 5), dtype=np.int32)
+    _check(lib.tlr_debug_plan_tiles(n, V, sm_count, mlp_hidden, c_void_p(out.ctypes.data), count.value, byref(count),
+                                    byref(plan)), "tlr_debug_plan_tiles")
     return out, plan
 
 

@@ -2,6 +2,7 @@
 #include <cuda.h>
 #include <cuda_runtime.h>
 
+#include <cstdio>
 #include <cstdlib>
 #include <cstring>
 #include <new>
@@ -16,17 +17,42 @@ namespace tlr {
 constexpr int kMaxChunks = 192;       // upper bound on partials per row (sizes the workspace)
 constexpr int kMaxTimedLaunches = 4096;
 
+const Tuning& tuning() {
+  static const Tuning t = [] {
+    Tuning v = {};
+    v.tc8_inline = 1;
+    if (const char* e = getenv("TLR_TC_GRANULE")) v.granule = atoi(e);
+    if (getenv("TLR_TC_EVEN_TILES") != nullptr) v.even_tiles = 1;
+    if (const char* e = getenv("TLR_TC_RINGS")) {
+      int a = 0, b = 0;
+      if (sscanf(e, "%d,%d", &a, &b) == 2) {
+        v.ring_a = a;
+        v.ring_b = b;
+      }
+    }
+    if (const char* e = getenv("TLR_TC8_INLINE")) v.tc8_inline = e[0] == '0' ? 0 : 1;
+    if (const char* e = getenv("TLR_FINISH_THREADS")) v.finish_threads = atoi(e);
+    return v;
+  }();
+  return t;
+}
+
 // Chooses the vocabulary decomposition: every unit gets the same number of tiles, and the
-// number of chunks minimises (waves of units) x (rows of the largest chunk + a fixed cost
-// per tile), so that workers finish together.
-void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
+// number of chunks minimises the load of the busiest worker -- (waves of units) x (rows of the
+// largest chunk + a fixed cost per tile) -- so that workers finish together.  With a learned
+// router in the launch (mlp_hidden > 0) one more unit per row unit, over the rows of its first
+// layer, follows the vocabulary units in the same round-robin order and is counted in the loads.
+void tc_plan(int n, int V, int cta, int workers, int max_chunks, int mlp_hidden, TcPlan* plan) {
   int g = 16 * cta;
-  if (const char* env = getenv("TLR_TC_GRANULE")) {   // tuning switch
-    const int e = atoi(env);
+  {
+    const int e = tuning().granule;   // tuning switch
     if (e >= g && e <= 256 && e % g == 0 && 256 % e == 0) g = e;
   }
   const int row_units = (n + 128 * cta - 1) / (128 * cta);
   const int granules = (V + g - 1) / g;
+  const int mlp_rows = mlp_hidden > 0 ? ((mlp_hidden + 16 * cta - 1) / (16 * cta)) * (16 * cta) : 0;
+  const long long mlp_tiles = (mlp_rows + 255) / 256;
+  const long long mlp_cost = mlp_rows + 24 * mlp_tiles;
   int hi = granules < max_chunks ? granules : max_chunks;
   if (hi < 1) hi = 1;
   long long best_cost = -1;
@@ -35,8 +61,23 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
     const long long gmax = (granules + c - 1) / c;
     const long long tiles = (gmax * g + 255) / 256;
     const long long units = 1ll * row_units * c;
-    const long long waves = (units + workers - 1) / workers;
-    const long long cost = waves * (gmax * g + 24 * tiles);
+    const long long unit_cost = gmax * g + 24 * tiles;
+    long long cost;
+    if (mlp_rows == 0) {
+      const long long waves = (units + workers - 1) / workers;
+      cost = waves * unit_cost;
+    } else {
+      // worker w takes units w, w + workers, ...: vocabulary units first, then the row_units router units
+      const long long full = units / workers, rem = units % workers;
+      cost = 0;
+      for (int w = 0; w < workers; ++w) {
+        const long long nv = full + (w < rem ? 1 : 0);
+        const long long j0 = ((w - rem) % workers + workers) % workers;   // first router unit of this worker
+        const long long nm = j0 < row_units ? 1 + (row_units - 1 - j0) / workers : 0;
+        const long long load = nv * unit_cost + nm * mlp_cost;
+        if (load > cost) cost = load;
+      }
+    }
     if (best_cost < 0 || cost < best_cost) {
       best_cost = cost;
       best = c;
@@ -48,17 +89,19 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, TcPlan* plan) {
   plan->granule_rows = g;
   plan->granules = granules;
   plan->tiles_per_unit = best_tiles;
+  plan->mlp_rows = mlp_rows;
   // How a unit's chunk is cut into tiles.  A tile costs a pass over all of h whatever its width,
   // so where the tensor pipe matters (pairs of CTAs, n > 128) the chunk is cut into full 256-row
   // tiles plus one remainder tile.  With one CTA per worker the path is HBM-bound and a narrow
   // remainder tile only lowers the bytes in flight, so the tiles are of equal size there.
   plan->full_tiles_first = 0;
-  if (cta == 2 && getenv("TLR_TC_EVEN_TILES") == nullptr) {   // (the variable is a tuning switch)
+  if (cta == 2 && !tuning().even_tiles) {   // (a tuning switch)
     const long long gmax = (granules + best - 1) / best;
     const long long full = 256 / g;
     plan->full_tiles_first = 1;
     plan->tiles_per_unit = static_cast<int>((gmax + full - 1) / full);
   }
+  if (plan->tiles_per_unit < mlp_tiles) plan->tiles_per_unit = static_cast<int>(mlp_tiles);
 }
 
 }  // namespace tlr
@@ -113,6 +156,26 @@ struct tlr_ctx {
   bool timing = false;
   std::vector<cudaEvent_t> events;   // pairs, created lazily
   int timed = 0;
+
+  // Everything a call needs that depends only on (n, learned router in the launch or not): planned once
+  // and kept, so that a repeated call does no planning, reads no environment variable and -- when h sits
+  // at the same address as last time -- encodes no tensor map.
+  struct Step {
+    int n = -1;
+    bool mlp = false;
+    tlr_plan plan;
+    tlr::TcConfig cfg;
+    tlr::TcParams params;     // all but the per-call fields
+    tlr::TcMaps maps;
+    const void* h_mapped = nullptr;   // the address maps.h was encoded for
+    int workers = 0;
+  };
+  static constexpr int kSteps = 8;
+  Step steps[kSteps];
+  int next_step = 0;
+  // learned router inside the projection launch: tensor maps over W1 (needs d % 8 == 0 and an aligned W1)
+  bool mlp_fused = false;
+  CUtensorMap map_m128, map_m64, map_m16;
 };
 
 namespace {
@@ -145,35 +208,76 @@ tlr_path pick_path(const tlr_ctx* c) {
   return c->tc_ok ? TLR_PATH_TC : TLR_PATH_SIMT;
 }
 
-void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
+void forget_steps(tlr_ctx* c) {
+  for (auto& st : c->steps) st.n = -1;
+}
+
+// Plans a call of n rows (with or without the learned router inside the projection launch).
+void plan_step(const tlr_ctx* c, int n, bool mlp, tlr_ctx::Step* st) {
   const tlr_path path = pick_path(c);
+  tlr_plan* out = &st->plan;
+  st->n = n;
+  st->mlp = mlp;
+  st->h_mapped = nullptr;
+  st->workers = 0;
   out->path = path;
   out->launches = n > 0 ? 2 : 1;
   out->reserved = 0;
-  if (c->fp8) {
-    tlr::Tc8Config cfg;
+  tlr::TcParams& p = st->params;
+  p = tlr::TcParams{};
+  if (c->fp8 || path == TLR_PATH_TC) {
+    tlr::TcConfig& cfg = st->cfg;
     tlr::TcPlan tp;
-    tlr::tc8_configure(n, c->d, &cfg);
-    tlr::tc_plan(n <= 128 ? n : 128, c->V, 1, c->sm_count, tlr::kMaxChunks, &tp);
-    out->vocab_chunks = tp.chunks;
-    out->row_units = 1;
-    out->grid = tp.chunks < c->sm_count ? tp.chunks : c->sm_count;
-    out->block = tlr::tc8_threads();
-    out->smem_bytes = cfg.smem_bytes;
-    out->launches = n > 0 ? (cfg.inline_split ? 2 : 3) : 1;
-  } else if (path == TLR_PATH_TC) {
-    tlr::TcConfig cfg;
-    tlr::TcPlan tp;
-    tlr::tc_configure(n, &cfg);
-    const int workers_max = c->sm_count / cfg.cta;
-    tlr::tc_plan(n, c->V, cfg.cta, workers_max, tlr::kMaxChunks, &tp);
-    const int units = tp.chunks * tp.row_units;
-    const int workers = units < workers_max ? units : workers_max;
+    int workers_max;
+    if (c->fp8) {
+      tlr::tc8_configure(n <= tlr::tc8_max_rows() ? n : tlr::tc8_max_rows(), c->d, &cfg);
+      workers_max = c->sm_count;
+      tlr::tc_plan(n <= 128 ? n : 128, c->V, 1, workers_max, tlr::kMaxChunks, 0, &tp);
+      out->launches = n > 0 ? (cfg.inline_split ? 2 : 3) : 1;
+    } else {
+      tlr::tc_configure(n, &cfg);
+      workers_max = c->sm_count / cfg.cta;
+      tlr::tc_plan(n, c->V, cfg.cta, workers_max, tlr::kMaxChunks, mlp ? c->mlp_hidden : 0, &tp);
+    }
+    const int units = (tp.chunks + (tp.mlp_rows > 0 ? 1 : 0)) * tp.row_units;
+    st->workers = units < workers_max ? units : workers_max;
     out->vocab_chunks = tp.chunks;
     out->row_units = tp.row_units;
-    out->grid = workers * cfg.cta;
+    out->grid = st->workers * cfg.cta;
     out->block = tlr::tc_threads();
     out->smem_bytes = cfg.smem_bytes;
+    p.n = n;
+    p.d = c->d;
+    p.V = c->V;
+    p.row_units = tp.row_units;
+    p.chunks = tp.chunks;
+    p.granules = tp.granules;
+    p.tiles_per_unit = tp.tiles_per_unit;
+    p.full_tiles_first = tp.full_tiles_first;
+    p.granule_rows = tp.granule_rows;
+    p.a_rows = cfg.a_rows;
+    p.part_rows = cfg.part_rows;
+    p.a_stages = cfg.a_stages;
+    p.b_stages = cfg.b_stages;
+    p.wait_limit_ns = c->debug_wait_ns;
+    p.debug_drop_w_copies = c->debug_kind == 1 ? 1 : 0;
+    p.w_wait = 0;
+    p.mlp_hidden = tp.mlp_rows > 0 ? c->mlp_hidden : 0;
+    p.mlp_rows = tp.mlp_rows;
+    p.mlp_b1 = c->mlp_b1;
+    p.mlp_w2 = c->mlp_w2;
+    p.mlp_out = c->mlp_scores;
+    p.inline_split = cfg.inline_split;
+    p.hscale = c->hscale;
+    p.wscale = c->wscale;
+    p.partials = c->partials;
+    p.status = c->status;
+    st->maps.w128 = c->map_w128;
+    st->maps.w64 = c->map_w64;
+    st->maps.w16 = c->map_w16;
+    st->maps.m128 = mlp ? c->map_m128 : c->map_w128;
+    st->maps.m64 = mlp ? c->map_m64 : c->map_w64;
+    st->maps.m16 = mlp ? c->map_m16 : c->map_w16;
   } else {
     int chunks, grid, block, smem;
     tlr::simt_plan(n, c->d, c->V, c->sm_count, &chunks, &grid, &block, &smem);
@@ -183,6 +287,16 @@ void fill_plan(const tlr_ctx* c, int n, tlr_plan* out) {
     out->block = block;
     out->smem_bytes = smem;
   }
+}
+
+// The kept plan of (n, mlp), planned now if it is not there (the oldest slot is reused).
+tlr_ctx::Step* step_for(tlr_ctx* c, int n, bool mlp) {
+  for (auto& st : c->steps)
+    if (st.n == n && st.mlp == mlp) return &st;
+  tlr_ctx::Step* st = &c->steps[c->next_step];
+  c->next_step = (c->next_step + 1) % tlr_ctx::kSteps;
+  plan_step(c, n, mlp, st);
+  return st;
 }
 
 void free_all(tlr_ctx* c) {
@@ -249,7 +363,7 @@ tlr_status new_context(int d, int V, const void* W_dev, int max_n, tlr_ctx** out
 }
 
 // Enqueues the projection kernel of a call with n > 0 rows: chunk partials into ctx->partials.
-tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const tlr_plan& plan, cudaStream_t stream) {
+tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, tlr_ctx::Step* st, cudaStream_t stream) {
   cudaEvent_t ev0 = nullptr, ev1 = nullptr;
   if (ctx->timing && ctx->timed < tlr::kMaxTimedLaunches) {
     const size_t need = 2 * static_cast<size_t>(ctx->timed + 1);
@@ -264,60 +378,22 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
   }
   cudaError_t e;
   if (ctx->fp8) {
-    tlr::Tc8Config cfg;
-    tlr::TcPlan tp;
-    tlr::tc8_configure(n, ctx->d, &cfg);
-    tlr::tc_plan(n, ctx->V, 1, ctx->sm_count, tlr::kMaxChunks, &tp);
+    const tlr::TcConfig& cfg = st->cfg;
     if (!cfg.inline_split &&
-        tlr::launch_h_split(h_bf16_dev, n, ctx->d, cfg.a_rows, ctx->h_parts, ctx->hscale, stream) != cudaSuccess)
+        tlr::launch_h_split(h_bf16_dev, n, ctx->d, cfg.part_rows, ctx->h_parts, ctx->hscale, stream) != cudaSuccess)
       return TLR_ERR_CUDA;
-    CUtensorMap map_h;
-    if (!make_map8(ctx, &map_h, ctx->h_parts, 2 * cfg.a_rows, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
-    tlr::Tc8Params p = {};
-    p.n = n;
-    p.d = ctx->d;
-    p.V = ctx->V;
-    p.chunks = tp.chunks;
-    p.granules = tp.granules;
-    p.tiles_per_unit = tp.tiles_per_unit;
-    p.granule_rows = tp.granule_rows;
-    p.a_rows = cfg.a_rows;
-    p.a_stages = cfg.a_stages;
-    p.b_stages = cfg.b_stages;
-    p.wait_limit_ns = ctx->debug_wait_ns;
-    p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
-    p.inline_split = cfg.inline_split;
-    p.h = h_bf16_dev;
-    p.hscale = ctx->hscale;
-    p.wscale = ctx->wscale;
-    p.partials = ctx->partials;
-    p.status = ctx->status;
-    e = tlr::launch_tc8_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid, stream);
-  } else if (plan.path == TLR_PATH_TC) {
-    tlr::TcConfig cfg;
-    tlr::TcPlan tp;
-    tlr::tc_configure(n, &cfg);
-    tlr::tc_plan(n, ctx->V, cfg.cta, ctx->sm_count / cfg.cta, tlr::kMaxChunks, &tp);
-    CUtensorMap map_h;
-    if (!make_map(ctx, &map_h, h_bf16_dev, n, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
-    tlr::TcParams p;
-    p.n = n;
-    p.d = ctx->d;
-    p.V = ctx->V;
-    p.row_units = tp.row_units;
-    p.chunks = tp.chunks;
-    p.granules = tp.granules;
-    p.tiles_per_unit = tp.tiles_per_unit;
-    p.full_tiles_first = tp.full_tiles_first;
-    p.granule_rows = tp.granule_rows;
-    p.a_rows = cfg.a_rows;
-    p.a_stages = cfg.a_stages;
-    p.b_stages = cfg.b_stages;
-    p.wait_limit_ns = ctx->debug_wait_ns;
-    p.debug_drop_w_copies = ctx->debug_kind == 1 ? 1 : 0;
-    p.partials = ctx->partials;
-    p.status = ctx->status;
-    e = tlr::launch_tc_projection(map_h, ctx->map_w128, ctx->map_w64, ctx->map_w16, p, cfg, plan.grid / cfg.cta, stream);
+    if (st->h_mapped != ctx->h_parts) {      // the two parts stacked: one box is the whole operand slab
+      if (!make_map8(ctx, &st->maps.h, ctx->h_parts, cfg.a_rows, ctx->d, cfg.a_rows)) return TLR_ERR_CUDA;
+      st->h_mapped = ctx->h_parts;
+    }
+    st->params.h = h_bf16_dev;
+    e = tlr::launch_tc8_projection(st->maps, st->params, cfg, st->workers, stream);
+  } else if (st->plan.path == TLR_PATH_TC) {
+    if (st->h_mapped != h_bf16_dev) {
+      if (!make_map(ctx, &st->maps.h, h_bf16_dev, n, ctx->d, st->cfg.a_rows)) return TLR_ERR_CUDA;
+      st->h_mapped = h_bf16_dev;
+    }
+    e = tlr::launch_tc_projection(st->maps, st->params, st->cfg, st->workers, stream);
   } else {
     tlr::SimtLaunch a;
     a.W = ctx->W;
@@ -325,7 +401,7 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, const 
     a.n = n;
     a.d = ctx->d;
     a.V = ctx->V;
-    a.chunks = plan.vocab_chunks;
+    a.chunks = st->plan.vocab_chunks;
     a.partials = ctx->partials;
     e = tlr::launch_simt_projection(a, stream);
   }
@@ -434,6 +510,8 @@ tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf1
     if (cudaMalloc(&ctx->mlp_scores, static_cast<size_t>(ctx->max_n) * blocks * sizeof(float)) != cudaSuccess) {
       cudaGetLastError();
       ctx->mlp_hidden = 0;
+      ctx->mlp_fused = false;
+      forget_steps(ctx);
       return TLR_ERR_NOMEM;
     }
     ctx->mlp_blocks_cap = blocks;
@@ -443,19 +521,29 @@ tlr_status tlr_set_router_mlp(tlr_ctx* ctx, int32_t d_hidden, const void* W1_bf1
   ctx->mlp_b1 = b1_dev;
   ctx->mlp_w2 = w2_dev;
   ctx->mlp_b2 = b2;
+  // Where the tensor-core kernel runs, W1's rows are walked by that kernel as one more unit per row unit
+  // (same staged h, same MMAs); that needs tensor maps over W1, i.e. 16-byte rows at a 16-byte aligned base.
+  ctx->mlp_fused = false;
+  if (ctx->tc_ok && !ctx->fp8 && ctx->d % 8 == 0 && (reinterpret_cast<uintptr_t>(W1_bf16_dev) & 15u) == 0 &&
+      make_map(ctx, &ctx->map_m128, W1_bf16_dev, d_hidden, ctx->d, 128) &&
+      make_map(ctx, &ctx->map_m64, W1_bf16_dev, d_hidden, ctx->d, 64) &&
+      make_map(ctx, &ctx->map_m16, W1_bf16_dev, d_hidden, ctx->d, 16))
+    ctx->mlp_fused = true;
+  forget_steps(ctx);
   return TLR_OK;
 }
 
-tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t* out, int32_t capacity,
-                                int32_t* count, tlr_plan* plan_out) {
-  if (n <= 0 || V <= 0 || sm_count < 2 || count == nullptr || capacity < 0 || (capacity > 0 && out == nullptr))
+tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t mlp_hidden, int32_t* out,
+                                int32_t capacity, int32_t* count, tlr_plan* plan_out) {
+  if (n <= 0 || V <= 0 || sm_count < 2 || mlp_hidden < 0 || count == nullptr || capacity < 0 ||
+      (capacity > 0 && out == nullptr))
     return TLR_ERR_ARG;
   tlr::TcConfig cfg;
   tlr::TcPlan tp;
   tlr::tc_configure(n, &cfg);
   const int workers_max = sm_count / cfg.cta;
-  tlr::tc_plan(n, V, cfg.cta, workers_max, tlr::kMaxChunks, &tp);
-  const int units = tp.chunks * tp.row_units;
+  tlr::tc_plan(n, V, cfg.cta, workers_max, tlr::kMaxChunks, mlp_hidden, &tp);
+  const int units = (tp.chunks + (tp.mlp_rows > 0 ? 1 : 0)) * tp.row_units;
   const int workers = units < workers_max ? units : workers_max;
   tlr::TcParams p = {};
   p.n = n;
@@ -466,6 +554,8 @@ tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t*
   p.tiles_per_unit = tp.tiles_per_unit;
   p.full_tiles_first = tp.full_tiles_first;
   p.granule_rows = tp.granule_rows;
+  p.mlp_hidden = tp.mlp_rows > 0 ? mlp_hidden : 0;
+  p.mlp_rows = tp.mlp_rows;
   *count = tlr::tc_enumerate_tiles(p, cfg.cta, workers, out, capacity);
   if (plan_out != nullptr) {
     plan_out->path = TLR_PATH_TC;
@@ -484,6 +574,7 @@ tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms) 
   if (ctx == nullptr || (kind != 0 && kind != 1)) return TLR_ERR_ARG;
   ctx->debug_kind = kind;
   ctx->debug_wait_ns = static_cast<unsigned long long>(wait_limit_ms) * 1000000ull;
+  forget_steps(ctx);
   return TLR_OK;
 }
 
@@ -493,13 +584,14 @@ tlr_status tlr_set_path(tlr_ctx* ctx, tlr_path path) {
   if (path == TLR_PATH_TC && !ctx->tc_ok) return TLR_ERR_UNSUPPORTED;
   if (path == TLR_PATH_SIMT && ctx->fp8) return TLR_ERR_UNSUPPORTED;
   ctx->forced = path;
+  forget_steps(ctx);
   return TLR_OK;
 }
 
 tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out) {
   if (ctx == nullptr || out == nullptr || n < 0) return TLR_ERR_ARG;
   if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
-  fill_plan(ctx, n, out);
+  *out = step_for(ctx, n, false)->plan;
   return TLR_OK;
 }
 
@@ -541,15 +633,17 @@ static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, fl
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
 
-  tlr_plan plan;
-  fill_plan(ctx, n, &plan);
+  // the learned router runs inside the projection launch wherever the tensor-core kernel of the bf16 head runs
+  const bool mlp_inside = want_mlp && ctx->mlp_fused && !ctx->fp8 && pick_path(ctx) == TLR_PATH_TC;
+  tlr_ctx::Step* st = step_for(ctx, n, mlp_inside);
+  const tlr_plan& plan = st->plan;
 
   if (n > 0) {
-    const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, plan, stream);
+    const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, st, stream);
     if (ps != TLR_OK) return ps;
   }
 
-  if (want_mlp && n > 0) {
+  if (want_mlp && !mlp_inside && n > 0) {
     tlr::MlpLaunch m;
     m.h = h_bf16_dev;
     m.W1 = ctx->mlp_W1;
@@ -569,7 +663,7 @@ static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, fl
   f.chunks = plan.vocab_chunks;
   f.tau = tau;
   f.mlp_partial = want_mlp ? ctx->mlp_scores : nullptr;
-  f.mlp_blocks = want_mlp ? tlr::mlp_hidden_blocks(ctx->mlp_hidden) : 0;
+  f.mlp_blocks = want_mlp ? (mlp_inside ? 1 : tlr::mlp_hidden_blocks(ctx->mlp_hidden)) : 0;
   f.mlp_b2 = ctx->mlp_b2;
   f.decide_on_mlp = (opt != nullptr && opt->score_source == TLR_SCORE_MLP) ? 1 : 0;
   f.mlp_score_out = opt != nullptr ? opt->mlp_score_dev : nullptr;
@@ -603,9 +697,9 @@ tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, in
   if (static_cast<long long>(v_offset) + ctx->V + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
   if (ctx->fp8 && n > tlr::tc8_max_rows()) return TLR_ERR_UNSUPPORTED;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  tlr_plan plan;
-  fill_plan(ctx, n, &plan);
-  const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, plan, stream);
+  tlr_ctx::Step* st = step_for(ctx, n, false);
+  const tlr_plan& plan = st->plan;
+  const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, st, stream);
   if (ps != TLR_OK) return ps;
   if (tlr::launch_shard_summary(ctx->partials, n, plan.vocab_chunks, v_offset, static_cast<Partial*>(summary_dev),
                                 stream) != cudaSuccess)

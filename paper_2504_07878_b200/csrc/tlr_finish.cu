@@ -17,9 +17,8 @@
 //              call's CTAs do not have to wait for the merge to leave their SMs.
 //   larger n   many blocks of 8 warps; the block that finishes last (fence + ticket
 //              counter, no spinning) compacts the flags of all rows.
-#include <cstdlib>
-
 #include "tlr_common.cuh"
+#include "tlr_tc.cuh"
 
 namespace tlr {
 
@@ -356,8 +355,8 @@ cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream) {
     };
     int threads = kSmallThreads;
     if ((a.chunks + lanes_for(512) - 1) / lanes_for(512) <= kPerLane) threads = 512;
-    if (const char* env = getenv("TLR_FINISH_THREADS")) {   // tuning switch
-      const int e = atoi(env);
+    {
+      const int e = tuning().finish_threads;   // tuning switch (TLR_FINISH_THREADS)
       if (e == 256 || e == 512 || e == 1024) threads = e;
     }
     const int L = lanes_for(threads);

@@ -75,8 +75,13 @@ tlr_status setup_device(int dev, DeviceSetup** out) {
           q == cudaDriverEntryPointSuccess)
         g_encode = reinterpret_cast<EncodeTiledFn>(fn);
     }
-    s.tc_ready = (g_encode != nullptr) && (tlr::tc_prepare() == cudaSuccess);
-    cudaGetLastError();
+    // The tensor-core kernel must be usable on such a device; if its set-up failed (a transient
+    // error), nothing is recorded and the next call tries again.
+    if (g_encode == nullptr || tlr::tc_prepare() != cudaSuccess) {
+      cudaGetLastError();
+      return TLR_ERR_CUDA;
+    }
+    s.tc_ready = true;
     s.ready = true;
   }
   *out = &s;
@@ -120,27 +125,36 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
   unsigned int* ticket = reinterpret_cast<unsigned int*>(s->scratch + kTicketOffset);
   uint32_t* status = status_dev != nullptr ? status_dev : reinterpret_cast<uint32_t*>(s->scratch + kStatusOffset);
 
-  // The ticket must start at zero; the partials are fully rewritten for the rows in use.
+  int chunks = 1;
+  tlr::TcConfig cfg;
+  tlr::TcPlan tp = {};
+  tlr::TcMaps maps;
+  int workers = 0;
+  const bool tc = d % 8 == 0;
+  if (n > 0 && tc) {
+    if (!s->tc_ready) return TLR_ERR_CUDA;   // no silent change of kernel
+    tlr::tc_configure(n, &cfg);
+    const int workers_max = s->sm_count / cfg.cta;
+    tlr::tc_plan(n, V, cfg.cta, workers_max, kStaticMaxChunks, 0, &tp);
+    chunks = tp.chunks;
+    const int units = tp.chunks * tp.row_units;
+    workers = units < workers_max ? units : workers_max;
+    if (!encode_map(&maps.h, h_bf16_dev, n, d, cfg.a_rows) || !encode_map(&maps.w128, W_bf16_dev, V, d, 128) ||
+        !encode_map(&maps.w64, W_bf16_dev, V, d, 64) || !encode_map(&maps.w16, W_bf16_dev, V, d, 16))
+      return TLR_ERR_CUDA;
+    maps.m128 = maps.w128;
+    maps.m64 = maps.w64;
+    maps.m16 = maps.w16;
+  }
+
+  // The ticket must start at zero; the partials are fully rewritten for the rows in use.  These two
+  // clears are enqueued only once nothing on the host can fail any more except the launches themselves.
   if (cudaMemsetAsync(ticket, 0, sizeof(unsigned int), stream) != cudaSuccess) return TLR_ERR_CUDA;
   if (cudaMemsetAsync(status, 0, sizeof(uint32_t), stream) != cudaSuccess) return TLR_ERR_CUDA;
 
-  int chunks = 1;
   if (n > 0) {
-    if (d % 8 == 0 && !s->tc_ready) return TLR_ERR_CUDA;   // no silent change of kernel
-    if (d % 8 == 0) {
-      tlr::TcConfig cfg;
-      tlr::TcPlan tp;
-      tlr::tc_configure(n, &cfg);
-      const int workers_max = s->sm_count / cfg.cta;
-      tlr::tc_plan(n, V, cfg.cta, workers_max, kStaticMaxChunks, &tp);
-      chunks = tp.chunks;
-      const int units = tp.chunks * tp.row_units;
-      CUtensorMap map_h, map_w128, map_w64, map_w16;
-      if (!encode_map(&map_h, h_bf16_dev, n, d, cfg.a_rows) || !encode_map(&map_w128, W_bf16_dev, V, d, 128) ||
-          !encode_map(&map_w64, W_bf16_dev, V, d, 64) ||
-          !encode_map(&map_w16, W_bf16_dev, V, d, 16))
-        return TLR_ERR_CUDA;
-      tlr::TcParams p;
+    if (tc) {
+      tlr::TcParams p = {};
       p.n = n;
       p.d = d;
       p.V = V;
@@ -151,15 +165,15 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
       p.full_tiles_first = tp.full_tiles_first;
       p.granule_rows = tp.granule_rows;
       p.a_rows = cfg.a_rows;
+      p.part_rows = cfg.part_rows;
       p.a_stages = cfg.a_stages;
       p.b_stages = cfg.b_stages;
-      p.wait_limit_ns = 0;
-      p.debug_drop_w_copies = 0;
+      // W is an argument of this call, so the kernel that precedes it in the stream may have written it:
+      // the W producer waits for that kernel like every other warp does.
+      p.w_wait = 1;
       p.partials = partials;
       p.status = status;
-      if (tlr::launch_tc_projection(map_h, map_w128, map_w64, map_w16, p, cfg, units < workers_max ? units : workers_max,
-                                    stream) != cudaSuccess)
-        return TLR_ERR_CUDA;
+      if (tlr::launch_tc_projection(maps, p, cfg, workers, stream) != cudaSuccess) return TLR_ERR_CUDA;
     } else {
       int grid, block, smem;
       tlr::simt_plan(n, d, V, s->sm_count, &chunks, &grid, &block, &smem);

@@ -13,9 +13,29 @@ from tests.parity import check_against_oracle, check_self_consistency, to_np
 pytestmark = pytest.mark.gpu
 
 
-def run_fp8(P, codes, scale, h_cpu, tau, max_n=None, **kw):
+class FullHead8:
+    """One full-size 8-bit head at a time: codes and scales on the host and the device, and the fp64 matrix
+    they stand for (1-2 GB)."""
+    key = None
+    codes_dev = scale_dev = w64 = None
+    host = None
+
+    @classmethod
+    def get(cls, d, V):
+        if cls.key != (d, V):
+            cls.codes_dev = cls.scale_dev = cls.w64 = cls.host = None
+            codes, scale = S.make_W8(d, V, seed=0)
+            cls.host = (codes, scale)
+            cls.w64 = O.dequantize_e4m3(codes.numpy(), scale.numpy())
+            cls.codes_dev, cls.scale_dev = codes.cuda(), scale.cuda()
+            cls.key = (d, V)
+        return cls.host
+
+
+def run_fp8(P, codes, scale, h_cpu, tau, max_n=None, on_device=False, **kw):
     n = h_cpu.shape[0]
-    r = P.Router(codes.cuda(), max_n=max(1, max_n or n), wscale=scale.cuda())
+    r = P.Router(codes if on_device else codes.cuda(), max_n=max(1, max_n or n),
+                 wscale=scale if on_device else scale.cuda())
     r.token.fill_(-7); r.conf.fill_(float("nan")); r.entropy.fill_(float("nan"))
     r.route_mask.fill_(9); r.routed_idx.fill_(-3); r.routed_count.fill_(-5)
     h = h_cpu.cuda() if n > 0 else torch.empty((0, codes.shape[1]), dtype=torch.bfloat16, device="cuda")
@@ -59,6 +79,33 @@ def test_fp8_head_matches_oracle_on_dequantised_matrix(pkg, n, d, V):
     assert gpu["plan"].launches == (2 if n <= 16 and d <= 1024 else 3)   # small batches of a small head: the kernel splits h itself
     check_self_consistency(gpu, tau, V)
     rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(h)), W64)
+    if rep["route_exempt_rows"] == 0:
+        assert gpu["routed_count"] == ref.routed_count
+        assert np.array_equal(gpu["routed_idx"][:ref.routed_count], ref.routed_idx)
+
+
+# The shapes the benchmark times with --fp8, in its launch configuration: the 0.5B-class head with 16 rows
+# (the kernel splits h itself) and the d = 2048 head of the batch sweep with 1 and 64 rows (separate split kernel,
+# shallower W ring).  Every row is compared with the oracle on the de-quantised matrix.
+FULL_SIZE = [("decode16", 16, True), ("sweep1", 1, False), ("sweep64", 64, False)]
+
+
+@pytest.mark.parametrize("name,n,inline", FULL_SIZE)
+def test_fp8_head_at_benchmark_sizes(pkg, name, n, inline):
+    wl = S.WORKLOADS[name]
+    assert wl.n == n
+    codes, scale = FullHead8.get(wl.d, wl.V)
+    W64 = FullHead8.w64
+    hid = S.make_h(n, wl.d, seed=0)
+    first = O.route_oracle(S.bf16_bits(hid.h), None, 0.5, W64=W64)
+    tau = O.percentile_tau(first.conf, 0.5) if n > 1 else 0.5
+    ref = O.with_threshold(first, tau)
+    gpu = run_fp8(pkg, FullHead8.codes_dev, FullHead8.scale_dev, hid.h, tau, on_device=True)
+    assert gpu["status"] == 0
+    assert gpu["plan"].launches == (2 if inline else 3)
+    assert gpu["plan"].grid >= 140                       # the whole GPU streams W, as in the benchmark
+    check_self_consistency(gpu, tau, wl.V)
+    rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), W64)
     if rep["route_exempt_rows"] == 0:
         assert gpu["routed_count"] == ref.routed_count
         assert np.array_equal(gpu["routed_idx"][:ref.routed_count], ref.routed_idx)

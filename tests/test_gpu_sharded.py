@@ -41,7 +41,9 @@ def run_sharded(P, W, h_cpu, tau, shards):
 
 
 @pytest.mark.parametrize("n,d,V,shards", [(16, 64, 3000, 2), (37, 128, 4099, 3), (200, 256, 20011, 4),
-                                          (300, 896, 9001, 8), (1, 64, 640, 2)])
+                                          (300, 896, 9001, 8), (1, 64, 640, 2),
+                                          # the benchmark's decode batch on the 0.5B-class head, eight shards
+                                          (256, 896, 151936, 8)])
 def test_sharded_matches_oracle_and_unsharded(pkg, n, d, V, shards):
     W = S.make_W(d, V, seed=n + V, std=0.1)
     hid = S.make_h(n, d, seed=n + V, W=W, planted_fraction=0.1 if n >= 16 else 0.0)

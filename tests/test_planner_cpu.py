@@ -58,5 +58,46 @@ def test_plan_argument_errors():
     import ctypes
     lib = P.load_library()
     c = ctypes.c_int32(0)
-    assert lib.tlr_debug_plan_tiles(0, 100, 148, None, 0, ctypes.byref(c), None) == 1
-    assert lib.tlr_debug_plan_tiles(10, 100, 148, None, 5, ctypes.byref(c), None) == 1
+    assert lib.tlr_debug_plan_tiles(0, 100, 148, 0, None, 0, ctypes.byref(c), None) == 1
+    assert lib.tlr_debug_plan_tiles(10, 100, 148, 0, None, 5, ctypes.byref(c), None) == 1
+    assert lib.tlr_debug_plan_tiles(10, 100, 148, -1, None, 0, ctypes.byref(c), None) == 1
+
+
+@pytest.mark.parametrize("n,V,hidden", [(16, 151936, 256), (256, 151936, 256), (300, 3001, 96), (8192, 151936, 256),
+                                        (64, 128256, 1000), (129, 5000, 40), (4096, 151936, 1024)])
+def test_learned_router_units_follow_the_vocabulary_units(n, V, hidden):
+    """With a learned router inside the launch its first layer's rows (reported as vocabulary rows V ..) are
+    walked once per row unit, by units numbered after all vocabulary units, and the vocabulary is still
+    covered exactly once."""
+    tiles, plan = P.tlr_debug_plan_tiles(n, V, 148, hidden)
+    g = plan.reserved
+    cta = 2 if n > 128 else 1
+    rows_per_unit = 128 * cta
+    vocab_units = plan.vocab_chunks * plan.row_units
+    assert np.array_equal(np.unique(tiles[:, 1]), np.arange(vocab_units + plan.row_units))
+    router = tiles[tiles[:, 1] >= vocab_units]
+    vocab = tiles[tiles[:, 1] < vocab_units]
+    assert np.all(vocab[:, 3] + vocab[:, 4] <= -(-V // g) * g) and np.all(router[:, 3] >= V)
+    padded = -(-hidden // (16 * cta)) * (16 * cta)
+    for ru in range(plan.row_units):
+        sel = router[router[:, 2] == ru * rows_per_unit]
+        assert len(np.unique(sel[:, 1])) == 1                      # one unit per row unit
+        order = np.argsort(sel[:, 3])
+        v0, rows = sel[order, 3] - V, sel[order, 4]
+        assert v0[0] == 0 and np.array_equal(v0[1:], (v0 + rows)[:-1]) and v0[-1] + rows[-1] == padded
+        assert np.all(rows % (16 * cta) == 0) and np.all(rows <= 256)
+        sel = vocab[vocab[:, 2] == ru * rows_per_unit]
+        order = np.argsort(sel[:, 3])
+        v0, rows = sel[order, 3], sel[order, 4]
+        assert v0[0] == 0 and np.array_equal(v0[1:], (v0 + rows)[:-1]) and V <= v0[-1] + rows[-1] < V + g
+    assert plan.grid <= 148
+
+
+def test_learned_router_costs_the_decode_plans_little():
+    """The busiest worker of the decode plans carries at most 3 % more rows with a 256-wide router inside."""
+    for n in (16, 256):
+        plain, _ = P.tlr_debug_plan_tiles(n, 151936, 148)
+        fused, _ = P.tlr_debug_plan_tiles(n, 151936, 148, 256)
+        a = np.bincount(plain[:, 0], weights=plain[:, 4]).max()
+        b = np.bincount(fused[:, 0], weights=fused[:, 4]).max()
+        assert b <= 1.03 * a
