@@ -73,10 +73,10 @@ void tc_configure(int n, TcConfig* c) {
 }
 
 cudaError_t tc_prepare() {
-  cudaError_t e = cudaFuncSetAttribute(tc_projection_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+  cudaError_t e = cudaFuncSetAttribute(tc_projection_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                        kSmemLimit);
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(tc_projection_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  return cudaFuncSetAttribute(tc_projection_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
 }
 
 cudaError_t launch_tc_projection(const TcMaps& maps, const TcParams& p, const TcConfig& c, int workers,
@@ -96,10 +96,10 @@ cudaError_t launch_tc_projection(const TcMaps& maps, const TcParams& p, const Tc
   cfg.attrs = attr;
   if (c.cta == 1) {
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1, false>, maps, p);
+    return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1>, maps, p);
   }
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2, false>, maps, p);
+  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<2>, maps, p);
 }
 
 }  // namespace tlr

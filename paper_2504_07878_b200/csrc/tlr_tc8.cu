@@ -19,12 +19,14 @@
 // bytes from HBM are half.
 //
 // This file holds what only the 8-bit head has: the split kernel, the shape of the launch and the
-// <1, true> instantiation of the projection kernel (tlr_tc_kernel.cuh; device helpers in tlr_tc8_dev.cuh).
+// launch of tc8_projection_kernel (the <1, true> instantiation of the projection kernel's body in
+// tlr_tc_kernel.cuh; device helpers in tlr_tc8_dev.cuh).
 #include <cuda.h>
 #include <cuda_bf16.h>
 
 #include "tlr_common.cuh"
 #include "tlr_tc.cuh"
+#define TLR_DEFINE_TC8_KERNEL
 #include "tlr_tc_kernel.cuh"
 
 namespace tlr {
@@ -77,7 +79,7 @@ void tc8_configure(int n, int d, TcConfig* c) {
   const int budget = kSmemLimit - 1024 - kBarrierBytes - kScratchBytes - extra;
   // n <= 16 and all of h (two parts) small enough: the kernel splits h itself and keeps it resident, one
   // launch less.  TLR_TC8_INLINE=0 is a tuning switch that keeps the separate split kernel.
-  bool inl = n <= 16 && k_slabs <= kMaxAStages && tuning().tc8_inline != 0;
+  bool inl = n <= 16 && k_slabs * 8 <= kSplitLanes * kSplitChunks && tuning().tc8_inline != 0;
   // ... and only while the resident copy leaves the W ring five stages: with four (d = 2048) what the
   // missing launch gains is lost again to the shallower ring
   if (inl && (budget - k_slabs * a_stage) / b_stage < 5) inl = false;
@@ -94,7 +96,7 @@ void tc8_configure(int n, int d, TcConfig* c) {
 }
 
 cudaError_t tc8_prepare() {
-  return cudaFuncSetAttribute(tc_projection_kernel<1, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
+  return cudaFuncSetAttribute(tc8_projection_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemLimit);
 }
 
 cudaError_t launch_h_split(const void* h_bf16, int n, int d, int part_rows, uint8_t* parts, float* hscale,
@@ -124,7 +126,7 @@ cudaError_t launch_tc8_projection(const TcMaps& maps, const TcParams& p, const T
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, tc_projection_kernel<1, true>, maps, p);
+  return cudaLaunchKernelEx(&cfg, tc8_projection_kernel, maps, p);
 }
 
 }  // namespace tlr

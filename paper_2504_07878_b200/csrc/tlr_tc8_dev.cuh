@@ -57,49 +57,65 @@ __device__ __forceinline__ void split_pair(float x0, float x1, uint16_t& p1, uin
   p2 = to_e4m3x2(x1 - f1.y, x0 - f1.x);
 }
 
-// Splits the (at most 16) rows of h into resident operand slabs, done by `threads` threads numbered t
-// (threads >= 256; the caller synchronises them with named barrier 1).  Slab ks is 32 rows of 128 bytes
+// Splits the (at most 16) rows of h into resident operand slabs, done by 288 threads numbered t (the caller's
+// warps 2..10; they synchronise among themselves with named barrier 1).  Slab ks is 32 rows of 128 bytes
 // with the 128-byte swizzle TMA would have produced: rows 0..15 hold the first parts, rows 16..31 the
-// second parts; the 16-byte chunk c of row r sits at position c ^ (r & 7).  hs_s[r] receives row r's scale.
+// second parts; the 16-byte chunk c of row r sits at position c ^ (r & 7).  hs_s[r] receives row r's scale
+// (hs_s[32 + r] is scratch).  One pass over h: 18 threads per row, each keeps its (at most kSplitChunks) chunks of
+// 16 elements in registers between the maximum and the conversion, so the row is read from memory once and all
+// loads are in flight together.
+constexpr int kSplitThreads = 288;
+constexpr int kSplitLanes = kSplitThreads / 16;       // threads per row
+constexpr int kSplitChunks = 6;                       // chunks of 16 elements per thread: d <= 16 * 18 * 6 = 1728
 __device__ __forceinline__ void split_h_resident(const __nv_bfloat16* __restrict__ hb, int n, int d, int k_slabs,
-                                                 unsigned char* slabs, float* hs_s, int t, int threads) {
-  if (t < 256) {                                            // 16 threads per row: the row's scale
-    const int r = t >> 4, l = t & 15;
-    float amax = 0.f;
-    if (r < n) {
-      for (int k = l * 8; k < d; k += 128) {
-        const uint4 v = __ldg(reinterpret_cast<const uint4*>(hb + static_cast<size_t>(r) * d + k));
-        const __nv_bfloat162* b2 = reinterpret_cast<const __nv_bfloat162*>(&v);
+                                                 unsigned char* slabs, float* hs_s, int t) {
+  const int r = t / kSplitLanes, l = t - r * kSplitLanes;
+  const int valid_chunks = d >> 4;                          // d is a multiple of 16
+  uint4 va[kSplitChunks], vb[kSplitChunks];
+  float amax = 0.f;
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-          const float2 f = __bfloat1622float2(b2[j]);
-          amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
-        }
-      }
+  for (int i = 0; i < kSplitChunks; ++i) {
+    const int c = l + kSplitLanes * i;
+    va[i] = make_uint4(0u, 0u, 0u, 0u);
+    vb[i] = va[i];
+    if (r < n && c < valid_chunks) {
+      const uint4* src = reinterpret_cast<const uint4*>(hb + static_cast<size_t>(r) * d + c * 16);
+      va[i] = __ldg(src);
+      vb[i] = __ldg(src + 1);
     }
-#pragma unroll
-    for (int off = 8; off > 0; off >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, off));
-    if (l == 0) hs_s[r] = split_scale(amax);
   }
-  asm volatile("bar.sync 1, %0;" ::"r"(threads) : "memory");   // only the splitting warps; nothing asynchronous is waited for
-  const int chunks_per_row = k_slabs * 8;
-  for (int item = t; item < 16 * chunks_per_row; item += threads) {
-    const int r = item / chunks_per_row, cc = item - r * chunks_per_row;
-    const int ks = cc >> 3, c = cc & 7, k0 = cc * 16;
-    uint32_t q1[4] = {0u, 0u, 0u, 0u}, q2[4] = {0u, 0u, 0u, 0u};
-    if (r < n && k0 < d) {                                  // d is a multiple of 16
-      const float inv = 1.0f / hs_s[r];                     // exact: a power of two
-      const uint4 va = __ldg(reinterpret_cast<const uint4*>(hb + static_cast<size_t>(r) * d + k0));
-      const uint4 vb = __ldg(reinterpret_cast<const uint4*>(hb + static_cast<size_t>(r) * d + k0 + 8));
-      const uint32_t w[8] = {va.x, va.y, va.z, va.w, vb.x, vb.y, vb.z, vb.w};
 #pragma unroll
-      for (int j = 0; j < 8; ++j) {                          // two elements per 32-bit word
-        const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[j]));
-        uint16_t p1, p2;
-        split_pair(f.x * inv, f.y * inv, p1, p2);
-        q1[j >> 1] |= static_cast<uint32_t>(p1) << (16 * (j & 1));
-        q2[j >> 1] |= static_cast<uint32_t>(p2) << (16 * (j & 1));
-      }
+  for (int i = 0; i < kSplitChunks; ++i) {
+    const uint32_t w[8] = {va[i].x, va[i].y, va[i].z, va[i].w, vb[i].x, vb[i].y, vb[i].z, vb[i].w};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[j]));
+      amax = fmaxf(amax, fmaxf(fabsf(f.x), fabsf(f.y)));
+    }
+  }
+  // the row's largest magnitude: non-negative floats order like their bit patterns
+  unsigned int* amax_bits = reinterpret_cast<unsigned int*>(hs_s + 32);
+  if (t < 16) amax_bits[t] = 0u;
+  asm volatile("bar.sync 1, %0;" ::"n"(kSplitThreads) : "memory");   // only the splitting warps; nothing asynchronous is waited for
+  atomicMax(amax_bits + r, __float_as_uint(amax));               // (fmaxf drops NaNs, so amax is a number >= 0)
+  asm volatile("bar.sync 1, %0;" ::"n"(kSplitThreads) : "memory");
+  const float sc = split_scale(__uint_as_float(amax_bits[r]));
+  if (l == 0) hs_s[r] = sc;
+  const float inv = 1.0f / sc;                                   // exact: a power of two
+#pragma unroll
+  for (int i = 0; i < kSplitChunks; ++i) {
+    const int cc = l + kSplitLanes * i;
+    if (cc >= k_slabs * 8) continue;                             // (chunks between d and the slab's end are zeros)
+    const int ks = cc >> 3, c = cc & 7;
+    const uint32_t w[8] = {va[i].x, va[i].y, va[i].z, va[i].w, vb[i].x, vb[i].y, vb[i].z, vb[i].w};
+    uint32_t q1[4] = {0u, 0u, 0u, 0u}, q2[4] = {0u, 0u, 0u, 0u};
+#pragma unroll
+    for (int j = 0; j < 8; ++j) {                                // two elements per 32-bit word
+      const float2 f = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162*>(&w[j]));
+      uint16_t p1, p2;
+      split_pair(f.x * inv, f.y * inv, p1, p2);
+      q1[j >> 1] |= static_cast<uint32_t>(p1) << (16 * (j & 1));
+      q2[j >> 1] |= static_cast<uint32_t>(p2) << (16 * (j & 1));
     }
     unsigned char* dst = slabs + ks * 4096 + r * 128 + ((c ^ (r & 7)) << 4);
     *reinterpret_cast<uint4*>(dst) = make_uint4(q1[0], q1[1], q1[2], q1[3]);

@@ -3,7 +3,7 @@
 // online-softmax reduction (max / argmax / sum-exp / entropy numerator) fused into
 // the epilogue, so the n x V logits never leave the SM.
 //
-// One kernel template, three instantiations:
+// One kernel body, three instantiations (two kernels at the end of this file):
 //   <1, false>  bf16 head, one CTA per worker, MMA M = 128 token rows     (n <= 128; M = 64 when n <= 64)
 //   <2, false>  bf16 head, a cluster of two CTAs per worker, MMA M = 256 rows (cta_group::2): each
 //               CTA stages its own 128 rows of h and HALF of the W tile, and the pair's
@@ -206,9 +206,10 @@ struct RowFold {
 
 }  // namespace
 
+// The kernel body (maps and p are the kernel's own parameters, maps a __grid_constant__ one: TMA reads the
+// tensor maps from parameter space).
 template <int kCta, bool kFp8>
-__global__ void __launch_bounds__(kThreads, 1)
-tc_projection_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+__device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcParams& p) {
   static_assert(!(kFp8 && kCta != 1), "the 8-bit head runs with one CTA per worker");
   extern __shared__ unsigned char smem_raw[];
   // 1024-byte alignment: the swizzle pattern is a function of the shared-memory address.
@@ -312,8 +313,8 @@ tc_projection_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
   if (inl && warp >= 2) {
     // ---- 8-bit head, n <= 16: the nine warps that have nothing to do yet split h into its two e4m3
     // parts, straight into the resident operand slabs
-    split_h_resident(static_cast<const __nv_bfloat16*>(p.h), p.n, p.d, k_slabs, gen_base, hs_s,
-                     threadIdx.x - 64, kThreads - 64);
+    static_assert(kThreads - 64 == kSplitThreads, "warps 2..10 split h");
+    split_h_resident(static_cast<const __nv_bfloat16*>(p.h), p.n, p.d, k_slabs, gen_base, hs_s, threadIdx.x - 64);
     __syncwarp();
     if (lane == 0) mbar_arrive(h_ready);
   }
@@ -609,5 +610,21 @@ tc_projection_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
     tmem_dealloc<kCta>(tmem_base, kTmemCols);
   }
 }
+
+// bf16 head: one CTA per worker (kCta = 1) or a pair (kCta = 2).
+template <int kCta>
+__global__ void __launch_bounds__(kThreads, 1)
+tc_projection_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+  tc_projection_body<kCta, false>(maps, p);
+}
+
+// 8-bit head (defined in the one file that launches it).  At most 128 registers per thread, so that a block of
+// the merge kernel (512 threads) fits on the SM beside this CTA and is resident, waiting, before this kernel ends.
+#ifdef TLR_DEFINE_TC8_KERNEL
+__global__ void __maxnreg__(128)
+tc8_projection_kernel(const __grid_constant__ TcMaps maps, const TcParams p) {
+  tc_projection_body<1, true>(maps, p);
+}
+#endif
 
 }  // namespace tlr
