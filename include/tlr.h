@@ -31,6 +31,7 @@
 #ifndef TLR_H_
 #define TLR_H_
 
+#include <stddef.h>
 #include <stdint.h>
 
 #ifdef __cplusplus
@@ -154,16 +155,19 @@ typedef struct {
 #define TLR_SCORE_MLP 1    /* the learned score of tlr_set_router_mlp */
 
 /*
- * tlr_set_router_mlp -- attach a learned router to the context.  The paper's deployed score is
- * "an MLP classifier which operates on the last-layer hidden state" (Sec. 3.1, Sec. 2.1) whose
- * width, activation and weights it does not give; the shape here is this library's assumption:
+ * tlr_set_router_mlp -- attach a learned router to the context.  The score the paper deploys is a
+ * small learned classifier (an MLP) fed with the last-layer hidden state (Sec. 3.1, Sec. 2.1); its
+ * width, activation and weights are not given, so the shape here is this library's assumption:
  *     score(h) = sigmoid( w2 . relu(W1 h + b1) + b2 )        in (0, 1), high = keep the small model
  *   d_hidden        hidden width, > 0
  *   W1_bf16_dev     bf16 [d_hidden, d] row-major on the device;  b1_dev, w2_dev  float [d_hidden];  b2 scalar
  * The pointers are BORROWED for the life of the context (or until replaced by another call).
  * Allocates ceil(d_hidden / 32) floats per max_n row for partial sums.  With a router attached, tlr_route_ex computes
- * the learned score of every row in one extra small kernel when opt->score_source == TLR_SCORE_MLP
- * or opt->mlp_score_dev != NULL; token, conf and entropy are produced as always.
+ * the learned score of every row when opt->score_source == TLR_SCORE_MLP or opt->mlp_score_dev != NULL; token, conf
+ * and entropy are produced as always.  Where the tensor-core projection kernel runs (bf16 head, d % 8 == 0, W1
+ * 16-byte aligned) the rows of W1 are walked by that same launch as one more work unit per 128 or 256 token rows --
+ * same staged hidden states, same MMAs, an epilogue that applies b1, ReLU and w2 and sums -- so the step keeps its
+ * two launches; otherwise one extra small kernel computes the score on CUDA cores.
  * Errors: TLR_ERR_ARG, TLR_ERR_NOMEM.  tlr_route_ex returns TLR_ERR_ARG when the learned score is
  * requested but no router is attached.
  */
@@ -201,6 +205,59 @@ tlr_status tlr_shard_summary(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, in
 tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t shards, int32_t n, float tau,
                             int32_t* token_dev, float* conf_dev, float* entropy_dev, uint8_t* route_mask_dev,
                             int32_t* routed_idx_dev, int32_t* routed_count_dev, void* cuda_stream);
+
+/*
+ * tlr_shard_attach / tlr_shard_push / tlr_shard_finish_fused -- the vocabulary-sharded step with the exchange
+ * fused into the kernels (the per-token decision of Sec. 3.1 sits on the decode critical path -- Table 1,
+ * "TBT for SLM" -- so at decode sizes the exchange latency is what sharding must not add back): instead of an
+ * all-gather between two calls, every GPU STORES its per-row summaries straight into a block of every peer's
+ * memory and then sets a flag there; the peer's merge kernel waits for the flags of all ranks.  Peer stores
+ * only: nothing is loaded from a peer, nothing is multicast.
+ *
+ * Each GPU owns one exchange block of tlr_shard_block_bytes(max_n, shards) bytes (max_n as given to tlr_create
+ * on every rank), 256-byte aligned, that all peers can write (peer-mapped or symmetric memory), ZEROED by its
+ * owner before the first call.  Layout: 2 x shards uint32 flags, padded to 256 bytes, then 2 x shards slots of
+ * max_n summaries of 16 bytes; the two sets alternate from call to call, so a rank that is one call ahead
+ * does not overwrite what a slower peer still reads.
+ *
+ * tlr_shard_attach   rank in [0, shards), shards <= 192; peer_block_dev is a HOST array of `shards` device
+ *                    pointers, entry g = GPU g's block as addressable from this GPU (entry `rank` = this GPU's
+ *                    own block).  Allocates four small pointer tables; resets the call counter.  The blocks are
+ *                    BORROWED for the life of the context.
+ * tlr_shard_push     projection over this rank's rows of W (context created on them; v_offset = index of its
+ *                    first row in the full vocabulary), then one kernel that folds the chunk partials into the
+ *                    per-row summaries, stores them into this rank's slot on every peer and, after a
+ *                    system-wide fence, sets this rank's flag on every peer to the call number.
+ * tlr_shard_finish_fused  waits until the flags of all ranks in this GPU's block hold the current call number
+ *                    (bounded: after 2 s -- or the limit given to tlr_debug_inject -- the kernel raises
+ *                    TLR_DEV_WAIT_TIMEOUT and finishes on what is there), then merges the summaries in place
+ *                    and produces the six outputs of tlr_route.
+ * Every rank makes the same sequence of calls with the same n: push, finish, push, finish, ...  Stream,
+ * ownership and error rules as tlr_route; only tlr_shard_attach allocates.
+ * Errors: TLR_ERR_ARG (also: not attached, or finish before the first push), TLR_ERR_ALIGN,
+ * TLR_ERR_TOO_MANY_ROWS, TLR_ERR_UNSUPPORTED, TLR_ERR_NOMEM, TLR_ERR_CUDA.
+ */
+size_t tlr_shard_block_bytes(int32_t max_n, int32_t shards);
+tlr_status tlr_shard_attach(tlr_ctx* ctx, int32_t rank, int32_t shards, void* const* peer_block_dev);
+tlr_status tlr_shard_push(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, int32_t v_offset, void* cuda_stream);
+tlr_status tlr_shard_finish_fused(tlr_ctx* ctx, int32_t n, float tau, int32_t* token_dev, float* conf_dev,
+                                  float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev,
+                                  int32_t* routed_count_dev, void* cuda_stream);
+
+/*
+ * tlr_rows_merge -- row-sharded batches (every GPU routes its own rows of a large batch with its own copy of
+ * W; positions are independent, Sec. 3.1): turns the ranks' routed-index lists into ONE ascending list of
+ * global row numbers.  gathered_idx_dev is int32 [ranks][cap] (slot g = rank g's routed_idx, as an all-gather
+ * with slots of `cap` entries delivers it), counts_dev int32 [ranks] (the ranks' routed_count) and
+ * row_offsets_dev int32 [ranks] (global number of rank g's first row; ascending with g).  Writes
+ * global_idx_dev[0 .. total) = the lists of rank 0, 1, ... back to back with each rank's offset added, and
+ * *global_count_dev = total = the sum of the counts.  global_idx_dev needs room for that sum (at most
+ * ranks * cap).  All device memory, caller-owned; needs no context; asynchronous on cuda_stream.
+ * Errors: TLR_ERR_ARG, TLR_ERR_CUDA.
+ */
+tlr_status tlr_rows_merge(const int32_t* gathered_idx_dev, const int32_t* counts_dev, const int32_t* row_offsets_dev,
+                          int32_t ranks, int32_t cap, int32_t* global_idx_dev, int32_t* global_count_dev,
+                          void* cuda_stream);
 
 /*
  * tlr_route_host -- the same step with HOST buffers: brings h to the device, runs
@@ -277,6 +334,14 @@ tlr_status tlr_debug_inject(tlr_ctx* ctx, int32_t kind, uint32_t wait_limit_ms);
  */
 tlr_status tlr_debug_plan_tiles(int32_t n, int32_t V, int32_t sm_count, int32_t mlp_hidden, int32_t* out,
                                 int32_t capacity, int32_t* count, tlr_plan* plan_out);
+
+/*
+ * tlr_debug_shard_table -- host-only: the addresses tlr_shard_attach derives for one rank and one parity of the
+ * call counter from the ranks' exchange-block addresses (no GPU needed; used by the CPU tests of the layout).
+ * slot_out[g] / flag_out[g] = where rank `rank` stores its summaries / its flag on peer g.
+ */
+tlr_status tlr_debug_shard_table(int32_t max_n, int32_t rank, int32_t shards, void* const* peer_block_dev,
+                                 int32_t parity, void** slot_out, void** flag_out);
 
 /* tlr_plan_query -- the launch plan a call with n rows would use.  No device work. */
 tlr_status tlr_plan_query(tlr_ctx* ctx, int32_t n, tlr_plan* out);

@@ -70,6 +70,18 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_shard_summary.restype = c_int32
     lib.tlr_shard_finish.argtypes = [P, P, c_int32, c_int32, c_float, P, P, P, P, P, P, P]
     lib.tlr_shard_finish.restype = c_int32
+    lib.tlr_shard_block_bytes.argtypes = [c_int32, c_int32]
+    lib.tlr_shard_block_bytes.restype = ctypes.c_size_t
+    lib.tlr_shard_attach.argtypes = [P, c_int32, c_int32, POINTER(P)]
+    lib.tlr_shard_attach.restype = c_int32
+    lib.tlr_shard_push.argtypes = [P, P, c_int32, c_int32, P]
+    lib.tlr_shard_push.restype = c_int32
+    lib.tlr_shard_finish_fused.argtypes = [P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_shard_finish_fused.restype = c_int32
+    lib.tlr_debug_shard_table.argtypes = [c_int32, c_int32, c_int32, POINTER(P), c_int32, POINTER(P), POINTER(P)]
+    lib.tlr_debug_shard_table.restype = c_int32
+    lib.tlr_rows_merge.argtypes = [P, P, P, c_int32, c_int32, P, P, P]
+    lib.tlr_rows_merge.restype = c_int32
     lib.tlr_destroy.argtypes = [P]
     lib.tlr_status_string.argtypes = [c_int32]
     lib.tlr_status_string.restype = c_char_p
@@ -169,6 +181,46 @@ def tlr_shard_finish(ctx, summaries, shards: int, n: int, tau: float, token, con
     _check(load_library().tlr_shard_finish(ctx, _ptr(summaries), shards, n, tau, _ptr(token), _ptr(conf),
                                            _ptr(entropy), _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
                                            _stream_handle(stream)), "tlr_shard_finish")
+
+
+def tlr_shard_block_bytes(max_n: int, shards: int) -> int:
+    """Size of one GPU's exchange block for the fused vocabulary-sharded step."""
+    return int(load_library().tlr_shard_block_bytes(max_n, shards))
+
+
+def tlr_shard_attach(ctx, rank: int, shards: int, peer_blocks):
+    """peer_blocks: `shards` device addresses (ints or tensors), entry g = GPU g's zeroed exchange block."""
+    arr = (c_void_p * shards)(*[_ptr(b) for b in peer_blocks])
+    _check(load_library().tlr_shard_attach(ctx, rank, shards, arr), "tlr_shard_attach")
+
+
+def tlr_debug_shard_table(max_n: int, rank: int, shards: int, peer_blocks, parity: int):
+    """Host-only: (slot addresses, flag addresses) of one rank on every peer, as tlr_shard_attach derives them."""
+    blocks = (c_void_p * shards)(*[_ptr(b) for b in peer_blocks])
+    slots, flags = (c_void_p * shards)(), (c_void_p * shards)()
+    _check(load_library().tlr_debug_shard_table(max_n, rank, shards, blocks, parity, slots, flags),
+           "tlr_debug_shard_table")
+    return [int(x or 0) for x in slots], [int(x or 0) for x in flags]
+
+
+def tlr_shard_push(ctx, h, n: int, v_offset: int, stream=None):
+    """Projection on this rank's shard, then the summaries stored into every peer's block and the flags set."""
+    _check(load_library().tlr_shard_push(ctx, _ptr(h), n, v_offset, _stream_handle(stream)), "tlr_shard_push")
+
+
+def tlr_shard_finish_fused(ctx, n: int, tau: float, token, conf, entropy, route_mask, routed_idx, routed_count,
+                           stream=None):
+    """Waits (bounded, on the device) for every rank's flag, then merges and decides like tlr_route."""
+    _check(load_library().tlr_shard_finish_fused(ctx, n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
+                                                 _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
+                                                 _stream_handle(stream)), "tlr_shard_finish_fused")
+
+
+def tlr_rows_merge(gathered_idx, counts, row_offsets, ranks: int, cap: int, global_idx, global_count, stream=None):
+    """Row-sharded batches: the ranks' routed-index lists [ranks][cap] -> one ascending list of global rows."""
+    _check(load_library().tlr_rows_merge(_ptr(gathered_idx), _ptr(counts), _ptr(row_offsets), ranks, cap,
+                                         _ptr(global_idx), _ptr(global_count), _stream_handle(stream)),
+           "tlr_rows_merge")
 
 
 def tlr_route_static(d: int, V: int, W, h, n: int, tau: float, token, conf, entropy, route_mask, routed_idx,

@@ -173,6 +173,13 @@ struct tlr_ctx {
   static constexpr int kSteps = 8;
   Step steps[kSteps];
   int next_step = 0;
+  // vocabulary-sharded step with the fused exchange (tlr_shard_attach): pointer tables on the device, one per
+  // parity of the call's epoch -- where this rank's summaries and flag go on every peer -- and this GPU's own block
+  int shard_rank = -1, shard_count = 0;
+  uint32_t shard_epoch = 0;
+  Partial** peer_slot[2] = {nullptr, nullptr};
+  uint32_t** peer_flag[2] = {nullptr, nullptr};
+  unsigned char* my_block = nullptr;
   // learned router inside the projection launch: tensor maps over W1 (needs d % 8 == 0 and an aligned W1)
   bool mlp_fused = false;
   CUtensorMap map_m128, map_m64, map_m16;
@@ -309,6 +316,10 @@ void free_all(tlr_ctx* c) {
   cudaFree(c->mlp_scores);
   cudaFree(c->h_parts);
   cudaFree(c->hscale);
+  for (int q = 0; q < 2; ++q) {
+    cudaFree(c->peer_slot[q]);
+    cudaFree(c->peer_flag[q]);
+  }
   for (cudaEvent_t e : c->events) cudaEventDestroy(e);
   delete c;
 }
@@ -657,10 +668,12 @@ static tlr_status route_step(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, fl
     if (tlr::launch_mlp_score(m, stream) != cudaSuccess) return TLR_ERR_CUDA;
   }
 
-  tlr::FinishLaunch f;
+  tlr::FinishLaunch f = {};
   f.partials = ctx->partials;
   f.n = n;
   f.chunks = plan.vocab_chunks;
+  f.row_stride = plan.vocab_chunks;
+  f.chunk_stride = 1;
   f.tau = tau;
   f.mlp_partial = want_mlp ? ctx->mlp_scores : nullptr;
   f.mlp_blocks = want_mlp ? (mlp_inside ? 1 : tlr::mlp_hidden_blocks(ctx->mlp_hidden)) : 0;
@@ -720,13 +733,12 @@ tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t sha
     if ((reinterpret_cast<uintptr_t>(summaries_dev) & 15u) != 0) return TLR_ERR_ALIGN;
   }
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
-  if (tlr::launch_shard_gather(static_cast<const Partial*>(summaries_dev), shards, n, ctx->partials, stream) !=
-      cudaSuccess)
-    return TLR_ERR_CUDA;
   tlr::FinishLaunch f = {};
-  f.partials = ctx->partials;
+  f.partials = static_cast<const Partial*>(summaries_dev);   // read in place: summary of shard g, row i at [g * n + i]
   f.n = n;
   f.chunks = shards;
+  f.row_stride = 1;
+  f.chunk_stride = n;
   f.tau = tau;
   f.token = token_dev;
   f.conf = conf_dev;
@@ -737,6 +749,149 @@ tlr_status tlr_shard_finish(tlr_ctx* ctx, const void* summaries_dev, int32_t sha
   f.ticket = ctx->ticket;
   f.status = ctx->status;
   if (tlr::launch_finish(f, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+// Layout of a GPU's exchange block for `shards` ranks and max_n rows: two sets (one per parity of the epoch) of
+// `shards` flags, padded to 256 bytes, then two sets of `shards` slots of max_n summaries.
+static size_t shard_header_bytes(int shards) { return (static_cast<size_t>(2) * shards * 4 + 255) & ~static_cast<size_t>(255); }
+
+size_t tlr_shard_block_bytes(int32_t max_n, int32_t shards) {
+  if (max_n <= 0 || shards <= 0) return 0;
+  return shard_header_bytes(shards) + static_cast<size_t>(2) * shards * max_n * sizeof(Partial);
+}
+
+tlr_status tlr_debug_shard_table(int32_t max_n, int32_t rank, int32_t shards, void* const* peer_block_dev,
+                                 int32_t parity, void** slot_out, void** flag_out) {
+  if (max_n <= 0 || shards < 1 || rank < 0 || rank >= shards || peer_block_dev == nullptr || slot_out == nullptr ||
+      flag_out == nullptr || (parity != 0 && parity != 1))
+    return TLR_ERR_ARG;
+  const size_t hdr = shard_header_bytes(shards);
+  const size_t np = static_cast<size_t>(max_n);
+  for (int g = 0; g < shards; ++g) {
+    unsigned char* base = static_cast<unsigned char*>(peer_block_dev[g]);
+    flag_out[g] = reinterpret_cast<uint32_t*>(base) + (static_cast<size_t>(parity) * shards + rank);
+    slot_out[g] = reinterpret_cast<Partial*>(base + hdr) + (static_cast<size_t>(parity) * shards + rank) * np;
+  }
+  return TLR_OK;
+}
+
+tlr_status tlr_shard_attach(tlr_ctx* ctx, int32_t rank, int32_t shards, void* const* peer_block_dev) {
+  if (ctx == nullptr || peer_block_dev == nullptr || shards < 1 || shards > tlr::kMaxChunks || rank < 0 ||
+      rank >= shards)
+    return TLR_ERR_ARG;
+  for (int g = 0; g < shards; ++g) {
+    if (peer_block_dev[g] == nullptr) return TLR_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(peer_block_dev[g]) & 255u) != 0) return TLR_ERR_ALIGN;
+  }
+  for (int q = 0; q < 2; ++q) {
+    cudaFree(ctx->peer_slot[q]);
+    cudaFree(ctx->peer_flag[q]);
+    ctx->peer_slot[q] = nullptr;
+    ctx->peer_flag[q] = nullptr;
+    std::vector<Partial*> slots(shards);
+    std::vector<uint32_t*> flags(shards);
+    if (tlr_debug_shard_table(ctx->max_n, rank, shards, peer_block_dev, q, reinterpret_cast<void**>(slots.data()),
+                              reinterpret_cast<void**>(flags.data())) != TLR_OK)
+      return TLR_ERR_ARG;
+    if (cudaMalloc(&ctx->peer_slot[q], shards * sizeof(Partial*)) != cudaSuccess ||
+        cudaMalloc(&ctx->peer_flag[q], shards * sizeof(uint32_t*)) != cudaSuccess) {
+      cudaGetLastError();
+      ctx->shard_count = 0;
+      return TLR_ERR_NOMEM;
+    }
+    if (cudaMemcpy(ctx->peer_slot[q], slots.data(), shards * sizeof(Partial*), cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(ctx->peer_flag[q], flags.data(), shards * sizeof(uint32_t*), cudaMemcpyHostToDevice) != cudaSuccess) {
+      ctx->shard_count = 0;
+      return TLR_ERR_CUDA;
+    }
+  }
+  ctx->shard_rank = rank;
+  ctx->shard_count = shards;
+  ctx->shard_epoch = 0;
+  ctx->my_block = static_cast<unsigned char*>(peer_block_dev[rank]);
+  return TLR_OK;
+}
+
+tlr_status tlr_shard_push(tlr_ctx* ctx, const void* h_bf16_dev, int32_t n, int32_t v_offset, void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || v_offset < 0 || ctx->shard_count == 0) return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n > 0) {
+    if (h_bf16_dev == nullptr) return TLR_ERR_ARG;
+    if ((reinterpret_cast<uintptr_t>(h_bf16_dev) & 15u) != 0) return TLR_ERR_ALIGN;
+  }
+  if (static_cast<long long>(v_offset) + ctx->V + 256 > 0x7fffffffll) return TLR_ERR_UNSUPPORTED;
+  if (ctx->fp8 && n > tlr::tc8_max_rows()) return TLR_ERR_UNSUPPORTED;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  int chunks = 1;
+  if (n > 0) {
+    tlr_ctx::Step* st = step_for(ctx, n, false);
+    chunks = st->plan.vocab_chunks;
+    const tlr_status ps = launch_projection(ctx, h_bf16_dev, n, st, stream);
+    if (ps != TLR_OK) return ps;
+  }
+  ctx->shard_epoch += 1;
+  if (ctx->shard_epoch == 0) ctx->shard_epoch = 2;    // (wrapped: keep the parity sequence, never publish 0)
+  const int q = static_cast<int>(ctx->shard_epoch & 1u);
+  tlr::ShardPush a;
+  a.partials = ctx->partials;
+  a.n = n;
+  a.chunks = chunks;
+  a.v_offset = v_offset;
+  a.shards = ctx->shard_count;
+  a.peer_slot = ctx->peer_slot[q];
+  a.peer_flag = ctx->peer_flag[q];
+  a.epoch = ctx->shard_epoch;
+  a.ticket = ctx->ticket;
+  if (tlr::launch_shard_push(a, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_shard_finish_fused(tlr_ctx* ctx, int32_t n, float tau, int32_t* token_dev, float* conf_dev,
+                                  float* entropy_dev, uint8_t* route_mask_dev, int32_t* routed_idx_dev,
+                                  int32_t* routed_count_dev, void* cuda_stream) {
+  if (ctx == nullptr || n < 0 || routed_count_dev == nullptr || ctx->shard_count == 0 || ctx->shard_epoch == 0)
+    return TLR_ERR_ARG;
+  if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
+  if (n > 0 && (token_dev == nullptr || conf_dev == nullptr || entropy_dev == nullptr || route_mask_dev == nullptr ||
+                routed_idx_dev == nullptr))
+    return TLR_ERR_ARG;
+  cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
+  const int q = static_cast<int>(ctx->shard_epoch & 1u);
+  const int G = ctx->shard_count;
+  const size_t np = static_cast<size_t>(ctx->max_n);
+  tlr::FinishLaunch f = {};
+  f.partials = reinterpret_cast<const Partial*>(ctx->my_block + shard_header_bytes(G)) + static_cast<size_t>(q) * G * np;
+  f.n = n;
+  f.chunks = G;
+  f.row_stride = 1;
+  f.chunk_stride = ctx->max_n;
+  f.wait_flags = reinterpret_cast<const uint32_t*>(ctx->my_block) + static_cast<size_t>(q) * G;
+  f.wait_count = G;
+  f.wait_value = ctx->shard_epoch;
+  f.wait_limit_ns = ctx->debug_wait_ns != 0 ? ctx->debug_wait_ns : 2000000000ull;
+  f.tau = tau;
+  f.token = token_dev;
+  f.conf = conf_dev;
+  f.entropy = entropy_dev;
+  f.route_mask = route_mask_dev;
+  f.routed_idx = routed_idx_dev;
+  f.routed_count = routed_count_dev;
+  f.ticket = ctx->ticket;
+  f.status = ctx->status;
+  if (tlr::launch_finish(f, stream) != cudaSuccess) return TLR_ERR_CUDA;
+  return TLR_OK;
+}
+
+tlr_status tlr_rows_merge(const int32_t* gathered_idx_dev, const int32_t* counts_dev, const int32_t* row_offsets_dev,
+                          int32_t ranks, int32_t cap, int32_t* global_idx_dev, int32_t* global_count_dev,
+                          void* cuda_stream) {
+  if (ranks < 1 || ranks > 65535 || cap < 0 || counts_dev == nullptr || row_offsets_dev == nullptr ||
+      global_count_dev == nullptr || (cap > 0 && (gathered_idx_dev == nullptr || global_idx_dev == nullptr)))
+    return TLR_ERR_ARG;
+  if (tlr::launch_rows_merge(gathered_idx_dev, counts_dev, row_offsets_dev, ranks, cap, global_idx_dev,
+                             global_count_dev, static_cast<cudaStream_t>(cuda_stream)) != cudaSuccess)
+    return TLR_ERR_CUDA;
   return TLR_OK;
 }
 

@@ -89,8 +89,16 @@ cudaError_t launch_simt_projection(const SimtLaunch& a, cudaStream_t stream);
 void simt_plan(int n, int d, int V, int sm_count, int* chunks, int* grid, int* block, int* smem);
 
 struct FinishLaunch {
-  const Partial* partials;  // [n][chunks]
+  const Partial* partials;  // partial j of row i at partials[i * row_stride + j * chunk_stride]
   int n, chunks;
+  int row_stride, chunk_stride;   // [n][chunks]: (chunks, 1); a block gathered shard-major [shards][rows]: (1, rows)
+  // optional: before reading the partials, wait until wait_flags[0 .. wait_count) all hold wait_value (flags that
+  // other GPUs set after storing their summaries into this GPU's memory); bounded by wait_limit_ns, after which
+  // TLR_DEV_WAIT_TIMEOUT is raised and the kernel goes on with what is there
+  const uint32_t* wait_flags;
+  int wait_count;
+  uint32_t wait_value;
+  unsigned long long wait_limit_ns;
   float tau;
   const float* mlp_partial;   // optional [n][mlp_blocks]: partial sums of the learned router's output layer
   int mlp_blocks;
@@ -117,7 +125,22 @@ cudaError_t launch_finish(const FinishLaunch& a, cudaStream_t stream);
 // and the gathered summaries [shards][n] laid out as partials [n][shards].
 cudaError_t launch_shard_summary(const Partial* partials, int n, int chunks, int v_offset, Partial* summary,
                                  cudaStream_t stream);
-cudaError_t launch_shard_gather(const Partial* gathered, int shards, int n, Partial* partials, cudaStream_t stream);
+// Fused exchange: the summaries are stored straight into slot `rank` of every peer's exchange block and, once all
+// rows are out, this rank's flag in every peer's flag array is set to `epoch` (peer stores only).
+struct ShardPush {
+  const Partial* partials;   // this shard's chunk partials [n][chunks]
+  int n, chunks, v_offset;
+  int shards;                // peers, this rank included
+  Partial* const* peer_slot; // device array [shards]: where this rank's n summaries go on peer g
+  uint32_t* const* peer_flag;  // device array [shards]: this rank's flag on peer g
+  uint32_t epoch;
+  unsigned int* ticket;      // zero before the launch; left zero
+};
+cudaError_t launch_shard_push(const ShardPush& a, cudaStream_t stream);
+// Row-sharded batches: the ranks' routed-index lists (slot g = rank g's list, `cap` entries each, the first
+// counts[g] valid) become one ascending list of global row numbers, idx + row_offset[g].
+cudaError_t launch_rows_merge(const int32_t* gathered_idx, const int32_t* counts, const int32_t* row_offsets,
+                              int ranks, int cap, int32_t* global_idx, int32_t* global_count, cudaStream_t stream);
 
 // Copy of `bytes` (a multiple of 16) from host memory the device can read directly to device
 // memory, done by a kernel so that the projection kernel behind it can be launched early.

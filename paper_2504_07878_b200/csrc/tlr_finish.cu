@@ -29,7 +29,7 @@ constexpr int kSmallRows = 1024;
 constexpr int kPerLane = 6;            // ceil(192 / 32): the most partials a lane can own
 
 // Folds one row's partials.  Every lane returns the same result.
-__device__ __forceinline__ Partial fold_row(const Partial* __restrict__ p, int chunks, int lane) {
+__device__ __forceinline__ Partial fold_row(const Partial* __restrict__ p, int chunks, int chunk_stride, int lane) {
   Partial q[kPerLane];
   float m = -INFINITY;
   int idx = kNoToken;
@@ -37,7 +37,7 @@ __device__ __forceinline__ Partial fold_row(const Partial* __restrict__ p, int c
   for (int k = 0; k < kPerLane; ++k) {
     const int j = lane + 32 * k;
     if (j < chunks) {
-      const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+      const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + static_cast<size_t>(j) * chunk_stride));
       q[k].m = raw.x;
       q[k].idx = __float_as_int(raw.y);
       q[k].s = raw.z;
@@ -135,6 +135,35 @@ __device__ __forceinline__ void pdl_enter() {
   asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
+// Vocabulary-sharded step with the fused exchange: the other GPUs store their summaries into this GPU's
+// memory and then set a flag each.  Warp 0 of every block polls the flags (lane g watches flag g, g + 32, ...)
+// with acquire loads at system scope until all hold the expected value or the time limit runs out; the
+// block then goes on either way (after a time-out the status word says the outputs are not to be trusted).
+__device__ __forceinline__ void wait_for_peers(const FinishLaunch& a) {
+  if (a.wait_flags == nullptr) return;
+  if (threadIdx.x < 32) {
+    unsigned long long t0 = 0;
+    asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t0));
+    for (;;) {
+      bool mine = true;
+      for (int g = threadIdx.x; g < a.wait_count; g += 32) {
+        uint32_t v;
+        asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(a.wait_flags + g) : "memory");
+        mine = mine && (v == a.wait_value);
+      }
+      if (__all_sync(0xffffffffu, mine)) break;
+      unsigned long long t1;
+      asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t1));
+      if (__any_sync(0xffffffffu, t1 - t0 > a.wait_limit_ns)) {
+        if (threadIdx.x == 0) atomicOr(a.status, TLR_DEV_WAIT_TIMEOUT);
+        break;
+      }
+      __nanosleep(200);
+    }
+  }
+  __syncthreads();
+}
+
 // Cluster of gridDim.x blocks, n <= 1024.  A group of L lanes (L a power of two) folds one
 // row in two passes over its partials: maximum and index first, then the sums rescaled to
 // that maximum.  L is chosen on the host so that every row has its group: n * L <=
@@ -147,12 +176,14 @@ finish_small_kernel(const FinishLaunch a, const int L) {
   const int group = (blockIdx.x * blockDim.x + threadIdx.x) / L;
   const int gl = threadIdx.x & (L - 1);
   pdl_enter();
+  wait_for_peers(a);
   __shared__ unsigned char flags[kSmallRows];
   const bool single_block = gridDim.x == 1;
   {
     const int row = group;
     const bool valid = row < a.n;
-    const Partial* p = a.partials + static_cast<size_t>(valid ? row : 0) * a.chunks;
+    const Partial* p = a.partials + static_cast<size_t>(valid ? row : 0) * a.row_stride;
+    const size_t cs = static_cast<size_t>(a.chunk_stride);
     float m = -INFINITY;
     int idx = kNoToken;
     float s = 0.f, t = 0.f;
@@ -163,7 +194,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
       for (int k = 0; k < kPerLane; ++k) {
         const int j = gl + L * k;
         if (valid && j < a.chunks) {
-          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j * cs));
           q[k].m = raw.x;
           q[k].idx = __float_as_int(raw.y);
           q[k].s = raw.z;
@@ -197,7 +228,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
       // many partials per lane: maximum and index first, then the rescaled sums
       if (valid) {
         for (int j = gl; j < a.chunks; j += L) {
-          const float2 mi = __ldcg(reinterpret_cast<const float2*>(p + j));
+          const float2 mi = __ldcg(reinterpret_cast<const float2*>(p + j * cs));
           const int qi = __float_as_int(mi.y);
           if (mi.x > m || (mi.x == m && qi < idx)) {
             m = mi.x;
@@ -215,7 +246,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
       }
       if (valid) {
         for (int j = gl; j < a.chunks; j += L) {
-          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j));
+          const float4 raw = __ldcg(reinterpret_cast<const float4*>(p + j * cs));
           if (!(raw.z == 0.f)) {
             const float dm = raw.x - m;
             const float e = exp2f(dm * kLog2e);
@@ -283,9 +314,10 @@ finish_kernel(const FinishLaunch a) {
   const int lane = threadIdx.x & 31;
   const int row = blockIdx.x * kFinishWarps + warp;
   pdl_enter();
+  wait_for_peers(a);
 
   if (row < a.n) {
-    const Partial acc = fold_row(a.partials + static_cast<size_t>(row) * a.chunks, a.chunks, lane);
+    const Partial acc = fold_row(a.partials + static_cast<size_t>(row) * a.row_stride, a.chunks, a.chunk_stride, lane);
     if (lane == 0) score_row(acc, a, row);
   }
 

@@ -193,6 +193,8 @@ extern "C" tlr_status tlr_route_static(int32_t d, int32_t V, const void* W_bf16_
   f.partials = partials;
   f.n = n;
   f.chunks = chunks;
+  f.row_stride = chunks;
+  f.chunk_stride = 1;
   f.tau = tau;
   f.mlp_partial = nullptr;
   f.mlp_blocks = 0;
