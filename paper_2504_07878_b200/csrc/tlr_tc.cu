@@ -20,15 +20,16 @@ int tc_enumerate_tiles(const TcParams& p, int cta, int workers, int* out, int ca
   const int units = (p.chunks + (p.mlp_hidden > 0 ? 1 : 0)) * p.row_units;
   for (int w = 0; w < workers; ++w) {
     for (int unit = w; unit < units; unit += workers) {
+      const Unit un = cta == 2 ? unit_of<2>(p, unit, 0) : unit_of<1>(p, unit, 0);
       for (int t = 0; t < p.tiles_per_unit; ++t) {
-        const Tile tl = cta == 2 ? tile_of<2>(p, unit, t, 0) : tile_of<1>(p, unit, t, 0);
+        const Tile tl = tile_of(p, un, t);
         if (tl.rows == 0) continue;
         if (count < capacity) {
           int* r = out + 5 * count;
           r[0] = w;
           r[1] = unit;
-          r[2] = tl.row0;
-          r[3] = tl.chunk < 0 ? p.V + tl.v0 : tl.v0;
+          r[2] = un.row0;
+          r[3] = un.chunk < 0 ? p.V + tl.v0 : tl.v0;
           r[4] = tl.rows;
         }
         ++count;

@@ -54,6 +54,8 @@
 #include <cuda.h>
 #include <cuda_bf16.h>
 
+#include <type_traits>
+
 #include "tlr_common.cuh"
 #include "tlr_tc.cuh"
 #include "tlr_tc8_dev.cuh"
@@ -86,44 +88,59 @@ __host__ __device__ constexpr int tc8_extra_bytes(int part_rows) {
 
 // The static schedule, identical in every role: worker w walks units w, w + workers, ...;
 // each unit is `tiles_per_unit` tiles (possibly empty ones when the chunk is short).
-struct Tile {
+struct Unit {
   int row0;    // first token row of this CTA in the unit
   int chunk;   // vocabulary chunk; -1 for a learned-router unit
+  int g0;      // first granule of the chunk
+  int G;       // granules in the chunk
+};
+struct Tile {
   int v0;      // first vocabulary row of the tile (first row of W1 in a learned-router unit)
   int rows;    // vocabulary rows in the tile (multiple of 16 * kCta); 0 = empty tile
 };
 
+// What is fixed for a whole unit (the divisions happen here, once per unit: the tile walk of the MMA-issuing
+// warp is on the tensor pipe's critical path and must stay cheap).
 template <int kCta>
-__host__ __device__ __forceinline__ Tile tile_of(const TcParams& p, int unit, int t, int cta_rank) {
-  Tile r;
+__host__ __device__ __forceinline__ Unit unit_of(const TcParams& p, int unit, int cta_rank) {
+  Unit u;
   const int vocab_units = p.chunks * p.row_units;
-  if (unit >= vocab_units) {
-    // learned-router unit: all rows of W1 for one row unit, in full 256-row tiles
-    r.chunk = -1;
-    r.row0 = ((unit - vocab_units) * kCta + cta_rank) * kBlockM;
+  if (unit >= vocab_units) {          // learned-router unit: all rows of W1 for one row unit
+    u.chunk = -1;
+    u.row0 = ((unit - vocab_units) * kCta + cta_rank) * kBlockM;
+    u.g0 = 0;
+    u.G = 0;
+    return u;
+  }
+  u.chunk = unit / p.row_units;
+  const int ru = unit - u.chunk * p.row_units;
+  u.row0 = (ru * kCta + cta_rank) * kBlockM;
+  u.g0 = static_cast<int>((static_cast<long long>(p.granules) * u.chunk) / p.chunks);
+  const int g1 = static_cast<int>((static_cast<long long>(p.granules) * (u.chunk + 1)) / p.chunks);
+  u.G = g1 - u.g0;
+  return u;
+}
+
+__host__ __device__ __forceinline__ Tile tile_of(const TcParams& p, const Unit& u, int t) {
+  Tile r;
+  if (u.chunk < 0) {                  // learned-router unit: full 256-row tiles over the rows of W1
     r.v0 = t * kBlockN;
     const int left = p.mlp_rows - r.v0;
     r.rows = left <= 0 ? 0 : (left < kBlockN ? left : kBlockN);
     return r;
   }
-  r.chunk = unit / p.row_units;
-  const int ru = unit - r.chunk * p.row_units;
-  r.row0 = (ru * kCta + cta_rank) * kBlockM;
-  const int g0 = static_cast<int>((static_cast<long long>(p.granules) * r.chunk) / p.chunks);
-  const int g1 = static_cast<int>((static_cast<long long>(p.granules) * (r.chunk + 1)) / p.chunks);
-  const int G = g1 - g0;
   int ga, gb;
   if (p.full_tiles_first) {
     // as many full 256-row tiles as fit, then one remainder tile: a tile costs a pass over all
     // of h whatever its width, so the fewest, widest tiles are the cheapest
     const int full = kBlockN / p.granule_rows;
-    ga = full * t < G ? full * t : G;
-    gb = full * (t + 1) < G ? full * (t + 1) : G;
+    ga = full * t < u.G ? full * t : u.G;
+    gb = full * (t + 1) < u.G ? full * (t + 1) : u.G;
   } else {
-    ga = (G * t) / p.tiles_per_unit;
-    gb = (G * (t + 1)) / p.tiles_per_unit;
+    ga = (u.G * t) / p.tiles_per_unit;
+    gb = (u.G * (t + 1)) / p.tiles_per_unit;
   }
-  r.v0 = (g0 + ga) * p.granule_rows;
+  r.v0 = (u.g0 + ga) * p.granule_rows;
   r.rows = (gb - ga) * p.granule_rows;
   return r;
 }
@@ -326,12 +343,13 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
       int slab = 0;     // running slab number, the same in every role
       bool ok = true;
       for (int unit = worker; unit < units && ok; unit += workers) {
+        const Unit un = unit_of<kCta>(p, unit, cta_rank);
         for (int t = 0; t < T && ok; ++t) {
-          const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+          const Tile tl = tile_of(p, un, t);
           if (tl.rows == 0) continue;
           const int my_rows = tl.rows / kCta;                 // this CTA's share of the tile
           const int my_v0 = tl.v0 + static_cast<int>(cta_rank) * my_rows;
-          const bool mlp = !kFp8 && tl.chunk < 0;
+          const bool mlp = !kFp8 && un.chunk < 0;
           const CUtensorMap* m128 = mlp ? &maps.m128 : &maps.w128;
           const CUtensorMap* m64p = mlp ? &maps.m64 : &maps.w64;
           const CUtensorMap* m16 = mlp ? &maps.m16 : &maps.w16;
@@ -365,8 +383,9 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
       int slab = 0;
       bool ok = true;
       for (int unit = worker; unit < units && ok; unit += workers) {
+        const Unit un = unit_of<kCta>(p, unit, cta_rank);
         for (int t = 0; t < T && ok; ++t) {
-          const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+          const Tile tl = tile_of(p, un, t);
           if (tl.rows == 0) continue;
           for (int ks = 0; ks < k_slabs; ++ks, ++slab) {
             if (slab >= SA) {
@@ -376,7 +395,7 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
             const uint32_t dst = a_ring + stage * a_stage_bytes;
             const uint32_t bar = (kCta == 2) ? map_to_cta(a_full(stage), 0) : a_full(stage);
             if (leader) mbar_expect_tx(a_full(stage), a_stage_bytes * kCta);
-            tma_load_2d<kCta>(dst, &maps.h, bar, ks * kSlabElems, kFp8 ? 0 : tl.row0);
+            tma_load_2d<kCta>(dst, &maps.h, bar, ks * kSlabElems, kFp8 ? 0 : un.row0);
             if (++stage == SA) stage = 0;
           }
         }
@@ -410,8 +429,9 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
       // issued, so the poll's latency overlaps the issue instead of adding to it.
       bool ra = inl || mbar_test_wait(a_full(0), 0), rb = mbar_test_wait(b_full(0), 0);
       for (int unit = worker; unit < units && ok; unit += workers) {
+        const Unit un = unit_of<kCta>(p, unit, 0);
         for (int t = 0; t < T && ok; ++t) {
-          const Tile tl = tile_of<kCta>(p, unit, t, 0);
+          const Tile tl = tile_of(p, un, t);
           if (tl.rows == 0) continue;
           const uint32_t idesc = kFp8 ? instr_desc_e4m3(mma_m, tl.rows) : instr_desc(mma_m, tl.rows);
           ok = __all_sync(0xffffffffu, mbar_wait(acc_empty(acc), acc_phase ^ 1u, abort_flag, p.status, wait_ns));
@@ -488,17 +508,21 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
     }
     if (kFp8) ok = __all_sync(0xffffffffu, ok);
     for (int unit = worker; unit < units && ok; unit += workers, ++ord) {
-      const Tile first = tile_of<kCta>(p, unit, 0, cta_rank);
+      const Unit first = unit_of<kCta>(p, unit, cta_rank);
       const bool warp_has_rows = !idle && (first.row0 + (m64 ? cquad * 16 : cquad * 32)) < p.n;   // warp-uniform
       const bool mlp_unit = !kFp8 && first.chunk < 0;
       RowFold f;
       f.reset();
       float mlp_sum = 0.f;
+      // The walk over the unit's tiles, compiled twice: once for vocabulary units (the hot loop, free of any
+      // learned-router code) and once for learned-router units.
+      auto walk_tiles = [&](auto router_tag) {
+      constexpr bool kRouter = decltype(router_tag)::value;
       for (int t = 0; t < T && ok; ++t) {
-        const Tile tl = tile_of<kCta>(p, unit, t, cta_rank);
+        const Tile tl = tile_of(p, first, t);
         if (tl.rows == 0) continue;
         const int v0 = tl.v0;
-        const int cols = min(tl.rows, (mlp_unit ? p.mlp_hidden : p.V) - v0);   // valid columns of this tile
+        const int cols = min(tl.rows, (kRouter ? p.mlp_hidden : p.V) - v0);   // valid columns of this tile
         // this group's share of them: [0, half) or [half, cols), half a multiple of 32
         const int half = min(cols, ((tl.rows / 2 + 31) / 32) * 32);
         const int c_begin = grp ? half : 0, c_end = grp ? cols : half;
@@ -548,7 +572,7 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
               if (lane == 0) mbar_arrive(hx_empty(hx));
               ++hx_n;
             }
-            if (mlp_unit) {
+            if constexpr (kRouter) {
               // hidden units v0 + c0 .. of the learned router: bias, ReLU, output-layer weight, sum
 #pragma unroll
               for (int j = 0; j < 32; ++j) {
@@ -572,6 +596,9 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
         }
         if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
       }
+      };
+      if (mlp_unit) walk_tiles(std::true_type{});
+      else walk_tiles(std::false_type{});
       if (donor || idle) continue;
       Partial out = f.result();
       if (mlp_unit) out.s = mlp_sum;
