@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc_kernel.cuh", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
-    "sha256": "06b0e7d9ace1da2464fade6a9fd2409357daa8602a903792937deb9dfb3c54ac",
-    "bytes_per_launch": {"decode256": 276.50e6, "decode16": 277.03e6, "sweep512": 531.47e6},
+    "sha256": "8f981209b227a46ae19d6a61e9ebc657ce578214267aa60cccf3d27c1aaf28d7",
+    "bytes_per_launch": {"decode256": 277.65e6, "decode16": 276.39e6, "sweep512": 532.87e6},
 }
 
 
@@ -294,7 +294,6 @@ def run_one_rank_of_a_vocab_shard(args):
     status = max(P.tlr_last_device_status(r.ctx) for r in ranks + mine[1:])
     if status & P.TLR_DEV_WAIT_TIMEOUT:
         raise SystemExit("device status flags raised: %d" % status)
-    ms = total_ms / steps
     peaks, peak_kind = measured_peaks()
     shard_bytes = 2 * (v1 - v0) * d + 2 * n * d + 17 * n + 4 + 16 * n * G
     print(json.dumps({"metric": METRIC, "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
