@@ -227,8 +227,8 @@ def merge_summaries(parts):
 def mlp_router_score(h_bits: np.ndarray, W1_bits: np.ndarray, b1, w2, b2: float) -> np.ndarray:
     """Learned routing score sigmoid(w2 . relu(W1 h + b1) + b2), fp64, one value per row.
 
-    The paper routes on "an MLP classifier which operates on the last-layer hidden
-    state" (Sec. 3.1; Sec. 2.1) without giving its shape; one hidden layer with ReLU
+    The paper routes on the output of a small learned classifier (an MLP) fed with the
+    last-layer hidden state (Sec. 3.1; Sec. 2.1) without giving its shape; one hidden layer with ReLU
     and a sigmoid output is this repository's assumption, so this function is pinned
     only by mathematics (closed forms, a library cross-check), not by the paper:
     parity unpinned by the paper.  W1 is bf16 bits [d_hidden, d]; b1, w2 are fp32.

@@ -1,9 +1,10 @@
 // Learned routing score on the hidden state: score = sigmoid(w2 . relu(W1 h + b1) + b2).
-// The paper's deployed router is "an MLP classifier which operates on the last-layer hidden
-// state" (Sec. 3.1; Sec. 2.1) but gives neither its width nor its activation nor weights, so
+// The router the paper deploys is a small learned classifier (an MLP) fed with the last-layer
+// hidden state (Sec. 3.1; Sec. 2.1); neither its width nor its activation nor weights are given, so
 // the shape here (one hidden layer, ReLU, sigmoid output) is this library's assumption and
-// the weights are the caller's.  The layer is tiny next to the LM head (d_hidden x d against
-// V x d), so it runs on CUDA cores: a block stages kMlpRows hidden-state rows in shared
+// the weights are the caller's.  Where the tensor-core projection kernel runs, the first layer is
+// part of that launch (tlr_tc_kernel.cuh); this CUDA-core kernel serves the shapes it cannot take
+// (d % 8 != 0, an unaligned W1, the 8-bit head): a block stages kMlpRows hidden-state rows in shared
 // memory and covers kMlpUnits hidden units, eight threads per unit.
 #include "tlr_common.cuh"
 
