@@ -84,7 +84,7 @@ typedef struct {
  *   max_n       largest n any later call will pass (>= 1).  Sizes the workspace.
  *   out         receives the context.
  * The only call that allocates device memory: the per-row partial-result workspace,
- * a status word, and staging buffers (device and pinned host) for tlr_route_host.  Uses the current CUDA device;
+ * a status word, and two sets of staging buffers (device and pinned host) for tlr_route_host.  Uses the current CUDA device;
  * every later call on the context must be made with that device current.
  * Errors: TLR_ERR_ARG, TLR_ERR_ALIGN, TLR_ERR_UNSUPPORTED (not an sm_100 device),
  * TLR_ERR_NOMEM, TLR_ERR_CUDA.  On error *out is NULL and nothing is leaked.
@@ -277,6 +277,24 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
                           int32_t* token_host, float* conf_host, float* entropy_host,
                           uint8_t* route_mask_host, int32_t* routed_idx_host,
                           int32_t* routed_count_host, void* cuda_stream);
+
+/*
+ * tlr_route_host_submit / tlr_route_host_collect -- tlr_route_host in two halves, so that a caller can keep TWO
+ * calls in flight: while the GPU works on one batch the host hands in the next, and the transfer of its hidden
+ * states over PCIe, the kernels' launch and the wake-up of the host overlap the previous batch's kernels
+ * (a serving loop that decodes for many sessions has the next batch ready before the last one is back).
+ *   submit   enqueues the copy of h to the device, the routing step and the write-back of its results into a
+ *            pinned block of the context, and returns without waiting.  h_bf16_host must stay valid and
+ *            unchanged until the matching collect has returned.  At most two submitted calls may be waiting to
+ *            be collected (a third returns TLR_ERR_ARG); all on one stream, or on streams the caller orders.
+ *   collect  waits for the OLDEST submitted call and hands out its results exactly as tlr_route_host does
+ *            (same optional pointers, same TLR_ERR_DEVICE_STATUS rule); TLR_ERR_ARG if none is waiting.
+ * tlr_route_host is submit followed by collect and returns TLR_ERR_ARG while submitted calls are waiting.
+ * Nothing is allocated (tlr_create sets up two staging slots).
+ */
+tlr_status tlr_route_host_submit(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau, void* cuda_stream);
+tlr_status tlr_route_host_collect(tlr_ctx* ctx, int32_t* token_host, float* conf_host, float* entropy_host,
+                                  uint8_t* route_mask_host, int32_t* routed_idx_host, int32_t* routed_count_host);
 
 /*
  * tlr_create_fp8 -- bind an 8-bit copy of the LM head for DECODE batches (the per-token step of

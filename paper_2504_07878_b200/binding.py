@@ -66,6 +66,10 @@ def load_library() -> ctypes.CDLL:
     lib.tlr_set_router_mlp.argtypes = [P, c_int32, P, P, P, c_float]
     lib.tlr_set_router_mlp.restype = c_int32
     lib.tlr_route_host.argtypes = [P, P, c_int32, c_float, P, P, P, P, P, P, P]
+    lib.tlr_route_host_submit.argtypes = [P, P, c_int32, c_float, P]
+    lib.tlr_route_host_submit.restype = c_int32
+    lib.tlr_route_host_collect.argtypes = [P, P, P, P, P, P, P]
+    lib.tlr_route_host_collect.restype = c_int32
     lib.tlr_shard_summary.argtypes = [P, P, c_int32, c_int32, P, P]
     lib.tlr_shard_summary.restype = c_int32
     lib.tlr_shard_finish.argtypes = [P, P, c_int32, c_int32, c_float, P, P, P, P, P, P, P]
@@ -167,6 +171,18 @@ def tlr_route_host(ctx, h, n: int, tau: float, token, conf, entropy, route_mask,
     _check(load_library().tlr_route_host(ctx, _ptr(h), n, tau, _ptr(token), _ptr(conf), _ptr(entropy),
                                          _ptr(route_mask), _ptr(routed_idx), _ptr(routed_count),
                                          _stream_handle(stream)), "tlr_route_host")
+
+
+def tlr_route_host_submit(ctx, h, n: int, tau: float, stream=None):
+    """First half of tlr_route_host: enqueue copy-in, step and write-back; h (a CPU tensor, ideally pinned) must stay
+    valid until the matching collect.  At most two submitted calls may be waiting."""
+    _check(load_library().tlr_route_host_submit(ctx, _ptr(h), n, tau, _stream_handle(stream)), "tlr_route_host_submit")
+
+
+def tlr_route_host_collect(ctx, token, conf, entropy, route_mask, routed_idx, routed_count):
+    """Second half: wait for the oldest submitted call and copy its results into the given CPU tensors."""
+    _check(load_library().tlr_route_host_collect(ctx, _ptr(token), _ptr(conf), _ptr(entropy), _ptr(route_mask),
+                                                 _ptr(routed_idx), _ptr(routed_count)), "tlr_route_host_collect")
 
 
 def tlr_shard_summary(ctx, h, n: int, v_offset: int, summary, stream=None):

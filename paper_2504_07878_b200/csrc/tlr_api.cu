@@ -129,10 +129,16 @@ struct tlr_ctx {
   // staging for tlr_route_host
   // One device block holds the six outputs of a call back to back, so that one copy brings
   // them all to a pinned host mirror: token[n] conf[n] entropy[n] routed_idx[n] count mask[n].
-  void* h_stage = nullptr;
-  unsigned char* out_stage = nullptr;    // device, 17 * max_n + 8 bytes
-  unsigned char* out_pinned = nullptr;   // pinned host mirror of the same size, + an aligned 4-byte status word
-  unsigned char* out_mapped = nullptr;   // the mirror as the device sees it (kernels write the results into it), or null
+  // Two slots, so that two host calls can be in flight (tlr_route_host_submit / _collect): slot s is used by
+  // every second call.
+  void* h_stage[2] = {nullptr, nullptr};
+  unsigned char* out_stage[2] = {nullptr, nullptr};    // device, 17 * max_n + 8 bytes
+  unsigned char* out_pinned[2] = {nullptr, nullptr};   // pinned host mirror of the same size, + an aligned 4-byte status word
+  unsigned char* out_mapped[2] = {nullptr, nullptr};   // the mirror as the device sees it (kernels write the results into it), or null
+  cudaEvent_t slot_done[2] = {nullptr, nullptr};       // recorded behind a submitted call's last kernel
+  int slot_n[2] = {0, 0};
+  int slot_next = 0;        // slot of the next submit
+  int slots_in_flight = 0;  // submitted and not yet collected (0..2); the oldest is slot (slot_next - in_flight) & 1
 
   // learned router (tlr_set_router_mlp)
   int mlp_hidden = 0;
@@ -168,6 +174,8 @@ struct tlr_ctx {
     tlr::TcParams params;     // all but the per-call fields
     tlr::TcMaps maps;
     const void* h_mapped = nullptr;   // the address maps.h was encoded for
+    const void* h_other = nullptr;    // ... and the address before that, with its map (two staging buffers alternate)
+    CUtensorMap h_other_map;
     int workers = 0;
   };
   static constexpr int kSteps = 8;
@@ -226,6 +234,7 @@ void plan_step(const tlr_ctx* c, int n, bool mlp, tlr_ctx::Step* st) {
   st->n = n;
   st->mlp = mlp;
   st->h_mapped = nullptr;
+  st->h_other = nullptr;
   st->workers = 0;
   out->path = path;
   out->launches = n > 0 ? 2 : 1;
@@ -310,9 +319,12 @@ void free_all(tlr_ctx* c) {
   cudaFree(c->partials);
   cudaFree(c->ticket);
   cudaFree(c->status);
-  cudaFree(c->h_stage);
-  cudaFree(c->out_stage);
-  cudaFreeHost(c->out_pinned);
+  for (int q = 0; q < 2; ++q) {
+    cudaFree(c->h_stage[q]);
+    cudaFree(c->out_stage[q]);
+    cudaFreeHost(c->out_pinned[q]);
+    if (c->slot_done[q] != nullptr) cudaEventDestroy(c->slot_done[q]);
+  }
   cudaFree(c->mlp_scores);
   cudaFree(c->h_parts);
   cudaFree(c->hscale);
@@ -346,17 +358,22 @@ tlr_status new_context(int d, int V, const void* W_dev, int max_n, tlr_ctx** out
   ok = ok && cudaMalloc(&c->partials, np * tlr::kMaxChunks * sizeof(Partial)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->ticket, sizeof(unsigned int)) == cudaSuccess;
   ok = ok && cudaMalloc(&c->status, sizeof(uint32_t)) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->h_stage, np * d * 2) == cudaSuccess;
-  ok = ok && cudaMalloc(&c->out_stage, np * 17 + 8) == cudaSuccess;
-  ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
+  for (int q = 0; q < 2; ++q) {
+    ok = ok && cudaMalloc(&c->h_stage[q], np * d * 2) == cudaSuccess;
+    ok = ok && cudaMalloc(&c->out_stage[q], np * 17 + 8) == cudaSuccess;
+    ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned[q]), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->slot_done[q], cudaEventDisableTiming) == cudaSuccess;
+  }
   if (!ok) {
     cudaGetLastError();
     free_all(c);
     return TLR_ERR_NOMEM;
   }
-  if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped), c->out_pinned, 0) != cudaSuccess) {
-    cudaGetLastError();
-    c->out_mapped = nullptr;   // tlr_route_host then stages the outputs in device memory and copies them
+  for (int q = 0; q < 2; ++q) {
+    if (cudaHostGetDevicePointer(reinterpret_cast<void**>(&c->out_mapped[q]), c->out_pinned[q], 0) != cudaSuccess) {
+      cudaGetLastError();
+      c->out_mapped[q] = nullptr;   // tlr_route_host then stages the outputs in device memory and copies them
+    }
   }
   if (cudaMemset(c->ticket, 0, sizeof(unsigned int)) != cudaSuccess ||
       cudaMemset(c->status, 0, sizeof(uint32_t)) != cudaSuccess) {
@@ -401,7 +418,17 @@ tlr_status launch_projection(tlr_ctx* ctx, const void* h_bf16_dev, int n, tlr_ct
     e = tlr::launch_tc8_projection(st->maps, st->params, cfg, st->workers, stream);
   } else if (st->plan.path == TLR_PATH_TC) {
     if (st->h_mapped != h_bf16_dev) {
-      if (!make_map(ctx, &st->maps.h, h_bf16_dev, n, ctx->d, st->cfg.a_rows)) return TLR_ERR_CUDA;
+      // the map in use moves to the second place; if that one was made for this address, it comes back
+      const void* was = st->h_mapped;
+      const CUtensorMap was_map = st->maps.h;
+      if (st->h_other == h_bf16_dev && h_bf16_dev != nullptr) {
+        st->maps.h = st->h_other_map;
+      } else if (!make_map(ctx, &st->maps.h, h_bf16_dev, n, ctx->d, st->cfg.a_rows)) {
+        st->h_mapped = nullptr;
+        return TLR_ERR_CUDA;
+      }
+      st->h_other = was;
+      st->h_other_map = was_map;
       st->h_mapped = h_bf16_dev;
     }
     e = tlr::launch_tc_projection(st->maps, st->params, st->cfg, st->workers, stream);
@@ -895,12 +922,12 @@ tlr_status tlr_rows_merge(const int32_t* gathered_idx_dev, const int32_t* counts
   return TLR_OK;
 }
 
-tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau, int32_t* token_host,
-                          float* conf_host, float* entropy_host, uint8_t* route_mask_host, int32_t* routed_idx_host,
-                          int32_t* routed_count_host, void* cuda_stream) {
-  if (ctx == nullptr || n < 0 || routed_count_host == nullptr) return TLR_ERR_ARG;
+tlr_status tlr_route_host_submit(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau, void* cuda_stream) {
+  if (ctx == nullptr || n < 0) return TLR_ERR_ARG;
   if (n > ctx->max_n) return TLR_ERR_TOO_MANY_ROWS;
   if (n > 0 && h_bf16_host == nullptr) return TLR_ERR_ARG;
+  if (ctx->slots_in_flight >= 2) return TLR_ERR_ARG;     // collect one first
+  const int q = ctx->slot_next;
   cudaStream_t stream = static_cast<cudaStream_t>(cuda_stream);
   const size_t nn = static_cast<size_t>(n);
   if (n > 0) {
@@ -916,22 +943,22 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
       mapped = attr.devicePointer;
     cudaGetLastError();
     if (mapped != nullptr) {
-      if (tlr::launch_host_copy(mapped, ctx->h_stage, bytes, stream) != cudaSuccess) return TLR_ERR_CUDA;
-    } else if (cudaMemcpyAsync(ctx->h_stage, h_bf16_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
+      if (tlr::launch_host_copy(mapped, ctx->h_stage[q], bytes, stream) != cudaSuccess) return TLR_ERR_CUDA;
+    } else if (cudaMemcpyAsync(ctx->h_stage[q], h_bf16_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
       return TLR_ERR_CUDA;
     }
   }
   // layout of the output block for this n (all offsets are multiples of 4)
   const size_t off_conf = 4 * nn, off_ent = 8 * nn, off_idx = 12 * nn, off_count = 16 * nn, off_mask = 16 * nn + 4;
   const size_t out_bytes = 17 * nn + 4;
-  unsigned char* pin = ctx->out_pinned;
+  unsigned char* pin = ctx->out_pinned[q];
   const size_t off_status = (static_cast<size_t>(ctx->max_n) * 17 + 8 + 3) & ~static_cast<size_t>(3);   // a 4-byte word
   uint32_t* pin_status = reinterpret_cast<uint32_t*>(pin + off_status);
   // The kernels write the six outputs and the status word straight into the pinned host block
   // (4 KB at n = 256); without a device view of it they go to device memory and are copied.
-  const bool direct = ctx->out_mapped != nullptr;
-  unsigned char* dev = direct ? ctx->out_mapped : ctx->out_stage;
-  const tlr_status st = route_step(ctx, ctx->h_stage, n, tau, nullptr, reinterpret_cast<int32_t*>(dev),
+  const bool direct = ctx->out_mapped[q] != nullptr;
+  unsigned char* dev = direct ? ctx->out_mapped[q] : ctx->out_stage[q];
+  const tlr_status st = route_step(ctx, ctx->h_stage[q], n, tau, nullptr, reinterpret_cast<int32_t*>(dev),
                                    reinterpret_cast<float*>(dev + off_conf), reinterpret_cast<float*>(dev + off_ent),
                                    dev + off_mask, reinterpret_cast<int32_t*>(dev + off_idx),
                                    reinterpret_cast<int32_t*>(dev + off_count), cuda_stream,
@@ -940,19 +967,48 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
   if (!direct && (cudaMemcpyAsync(pin, dev, out_bytes, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
                   cudaMemcpyAsync(pin_status, ctx->status, 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess))
     return TLR_ERR_CUDA;
-  if (cudaStreamSynchronize(stream) != cudaSuccess) return TLR_ERR_CUDA;
+  if (cudaEventRecord(ctx->slot_done[q], stream) != cudaSuccess) return TLR_ERR_CUDA;
+  ctx->slot_n[q] = n;
+  ctx->slot_next = q ^ 1;
+  ctx->slots_in_flight += 1;
+  return TLR_OK;
+}
+
+tlr_status tlr_route_host_collect(tlr_ctx* ctx, int32_t* token_host, float* conf_host, float* entropy_host,
+                                  uint8_t* route_mask_host, int32_t* routed_idx_host, int32_t* routed_count_host) {
+  if (ctx == nullptr || routed_count_host == nullptr || ctx->slots_in_flight <= 0) return TLR_ERR_ARG;
+  const int q = (ctx->slot_next - ctx->slots_in_flight) & 1;     // the oldest call in flight
+  if (cudaEventSynchronize(ctx->slot_done[q]) != cudaSuccess) return TLR_ERR_CUDA;
+  ctx->slots_in_flight -= 1;
+  const size_t nn = static_cast<size_t>(ctx->slot_n[q]);
+  const size_t off_conf = 4 * nn, off_ent = 8 * nn, off_idx = 12 * nn, off_count = 16 * nn, off_mask = 16 * nn + 4;
+  const unsigned char* pin = ctx->out_pinned[q];
+  const size_t off_status = (static_cast<size_t>(ctx->max_n) * 17 + 8 + 3) & ~static_cast<size_t>(3);
   int32_t count = 0;
   memcpy(&count, pin + off_count, 4);
   *routed_count_host = count;
-  if (n > 0) {
+  if (nn > 0) {
     if (token_host) memcpy(token_host, pin, 4 * nn);
     if (conf_host) memcpy(conf_host, pin + off_conf, 4 * nn);
     if (entropy_host) memcpy(entropy_host, pin + off_ent, 4 * nn);
     if (route_mask_host) memcpy(route_mask_host, pin + off_mask, nn);
     if (routed_idx_host && count > 0) memcpy(routed_idx_host, pin + off_idx, 4 * static_cast<size_t>(count));
   }
-  if (*pin_status & TLR_DEV_WAIT_TIMEOUT) return TLR_ERR_DEVICE_STATUS;
+  uint32_t status = 0;
+  memcpy(&status, pin + off_status, 4);
+  if (status & TLR_DEV_WAIT_TIMEOUT) return TLR_ERR_DEVICE_STATUS;
   return TLR_OK;
+}
+
+tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, float tau, int32_t* token_host,
+                          float* conf_host, float* entropy_host, uint8_t* route_mask_host, int32_t* routed_idx_host,
+                          int32_t* routed_count_host, void* cuda_stream) {
+  if (ctx == nullptr || routed_count_host == nullptr) return TLR_ERR_ARG;
+  if (ctx->slots_in_flight != 0) return TLR_ERR_ARG;     // not while submitted calls are waiting to be collected
+  const tlr_status st = tlr_route_host_submit(ctx, h_bf16_host, n, tau, cuda_stream);
+  if (st != TLR_OK) return st;
+  return tlr_route_host_collect(ctx, token_host, conf_host, entropy_host, route_mask_host, routed_idx_host,
+                                routed_count_host);
 }
 
 tlr_status tlr_last_device_status(tlr_ctx* ctx, uint32_t* out_host) {

@@ -29,6 +29,10 @@ host_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t 
     dst[i + 3 * stride] = d;
   }
   for (; i < n16; i += stride) dst[i] = src[i];
+  // Nothing above depends on the previous kernel in the stream (two staging buffers alternate between calls),
+  // but this kernel must not be complete before that one is: the projection kernel behind it waits for THIS
+  // kernel only, and it reuses the workspace the previous call's merge kernel reads.
+  asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 
 }  // namespace

@@ -197,6 +197,59 @@ def test_host_buffer_entry_point(pkg, how, n, d, V):
     pkg.tlr_destroy(ctx)
 
 
+def test_two_host_calls_in_flight(pkg):
+    """submit / collect: batches of different sizes are handed in while earlier ones are still on the GPU; every
+    collect returns the oldest call's results, which must be the oracle's for THAT batch."""
+    d, V = 256, 9001
+    W, _ = small_case(8, d, V, seed=12, planted=0.0)
+    Wd = W.cuda()
+    sizes = [300, 40, 129, 1, 300, 0, 64]                 # pair kernel, one-CTA kernels, an empty batch
+    batches = [S.make_h(n, d, seed=20 + i, W=W, planted_fraction=0.2 if n >= 5 else 0.0).h.pin_memory()
+               for i, n in enumerate(sizes)]
+    refs = [O.route_oracle(S.bf16_bits(b), S.bf16_bits(W), 0.5) if b.shape[0] else None for b in batches]
+    ctx = pkg.tlr_create(d, V, Wd, max(sizes))
+    m = max(sizes)
+    outs = lambda: (torch.empty(m, dtype=torch.int32).pin_memory(), torch.empty(m).pin_memory(), torch.empty(m).pin_memory(),
+                    torch.empty(m, dtype=torch.uint8).pin_memory(), torch.full((m,), -1, dtype=torch.int32).pin_memory(),
+                    torch.full((1,), -9, dtype=torch.int32).pin_memory())
+
+    def check(i, o):
+        n = sizes[i]
+        if n == 0:
+            assert int(o[5].item()) == 0
+            return
+        gpu = {"token": o[0].numpy()[:n], "conf": o[1].numpy()[:n], "entropy": o[2].numpy()[:n],
+               "route_mask": o[3].numpy()[:n], "routed_idx": o[4].numpy(), "routed_count": int(o[5].item())}
+        rep = check_against_oracle(refs[i], gpu)
+        check_self_consistency(gpu, 0.5, V)
+        if rep["route_exempt_rows"] == 0:
+            assert gpu["routed_count"] == refs[i].routed_count
+            assert np.array_equal(gpu["routed_idx"][:refs[i].routed_count], refs[i].routed_idx)
+
+    pkg.tlr_route_host_submit(ctx, batches[0], sizes[0], 0.5)
+    for i in range(1, len(sizes)):
+        pkg.tlr_route_host_submit(ctx, batches[i], sizes[i], 0.5)          # two in flight now
+        with pytest.raises(pkg.TlrError) as e:
+            pkg.tlr_route_host_submit(ctx, batches[i], sizes[i], 0.5)      # a third is refused
+        assert e.value.code == 1
+        o = outs()
+        pkg.tlr_route_host_collect(ctx, *o)
+        check(i - 1, o)
+    with pytest.raises(pkg.TlrError):                                      # the one-call form is refused meanwhile
+        pkg.tlr_route_host(ctx, batches[0], sizes[0], 0.5, *outs())
+    o = outs()
+    pkg.tlr_route_host_collect(ctx, *o)
+    check(len(sizes) - 1, o)
+    with pytest.raises(pkg.TlrError) as e:
+        pkg.tlr_route_host_collect(ctx, *outs())                           # nothing left to collect
+    assert e.value.code == 1
+    o = outs()
+    pkg.tlr_route_host(ctx, batches[2], sizes[2], 0.5, *o)                 # and the one-call form works again
+    check(2, o)
+    assert pkg.tlr_last_device_status(ctx) == 0
+    pkg.tlr_destroy(ctx)
+
+
 def test_argument_errors(pkg):
     W, hid = small_case(4, 64, 500, seed=1)
     Wd = W.cuda()
