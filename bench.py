@@ -583,6 +583,57 @@ def vocab_sharded_record(P, W_host, h_cpu, tau, rank, world, steps, warmup):
             "exchange": "NCCL all-gather of %d bytes per rank per step" % (16 * n)}
 
 
+def run_torch_eager(args):
+    """--impl torch-eager: what the step costs when written with library calls -- cuBLAS for the logits (written to
+    HBM), then torch's softmax, max, entropy, compare and nonzero.  Context beside the fused kernels, not a target
+    and not the reference arm; one GPU."""
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    if not torch.cuda.is_available():
+        raise SystemExit("needs a CUDA device")
+    torch.cuda.set_device(0)
+    wl = S.WORKLOADS[args.workload]
+    n, d, V = wl.n, wl.d, wl.V
+    tau = 0.5 if wl.tau is None else wl.tau
+    W_host = S.make_W(d, V, seed=0)
+    Ws = [W_host.cuda() for _ in range(2)]
+    h = S.make_h(n, d, seed=0, W=W_host, planted_fraction=wl.planted_fraction).h.cuda()
+
+    def step(i):
+        z = torch.matmul(h, Ws[i % 2].t()).float()
+        p = torch.softmax(z, dim=-1)
+        conf, token = p.max(dim=-1)
+        entropy = -(p * torch.log(p.clamp_min(1e-38))).sum(dim=-1)
+        mask = conf < tau
+        idx = torch.nonzero(mask).squeeze(-1)
+        return token, conf, entropy, mask, idx
+
+    def gemm_only(i):
+        return torch.matmul(h, Ws[i % 2].t())
+
+    def timed(fn, steps):
+        for i in range(max(3, args.warmup)):
+            fn(i)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    steps = min(args.steps, 2000 if n <= 256 else 100)
+    ms = timed(step, steps)
+    ms_gemm = timed(gemm_only, steps)
+    print(json.dumps({"impl": "torch-eager", "metric": METRIC, "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1,
+                      "steps": steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True,
+                      "scaling": "weak", "vs_baseline": None, "dtype": "bf16 GEMM (cuBLAS), fp32 softmax", "data": "synthetic",
+                      "config": {"workload": "%s: n=%d rows, d=%d, V=%d, tau=%g" % (wl.name, n, d, V, tau),
+                                 "what": "torch.matmul + softmax + max + entropy + compare + nonzero, logits in HBM"},
+                      "gemm_only_ms": ms_gemm, "gpu_launches": 0}))
+
+
 def blas_threads():
     try:
         from threadpoolctl import threadpool_info
@@ -661,7 +712,7 @@ def main():
     ap.add_argument("--steps", type=int, default=4000)
     ap.add_argument("--warmup", type=int, default=50)
     ap.add_argument("--workload", default="decode256", choices=sorted(S.WORKLOADS))
-    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference", "torch-eager"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extras", dest="extras", action="store_false",
                     help="default workload only: skip the sustained-load record and the decode16 / prefill8192 / "
@@ -682,7 +733,9 @@ def main():
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
-    if args.impl == "reference":
+    if args.impl == "torch-eager":
+        run_torch_eager(args)
+    elif args.impl == "reference":
         run_reference(args)
     elif args.one_shard_of > 1:
         run_one_rank_of_a_vocab_shard(args)

@@ -137,3 +137,52 @@ def test_learned_router_score(pkg, n, d, dh):
     torch.cuda.synchronize()
     assert np.array_equal(r.route_mask[:n].cpu().numpy(), base.route_mask)
     r.close()
+
+
+def test_learned_router_on_the_8bit_head_and_in_a_graph(pkg):
+    """Two more places the learned score must be right: on the 8-bit head (where the first layer runs in its own
+    kernel, the projection kernel multiplying e4m3 operands only) and inside a captured CUDA graph (where it is part
+    of the projection launch)."""
+    n, d, dh, V = 40, 128, 64, 3000
+    hid = S.make_h(n, d, seed=9)
+    g = torch.Generator().manual_seed(7)
+    W1 = (torch.randn(dh, d, generator=g) / d ** 0.5).to(torch.bfloat16)
+    b1 = torch.randn(dh, generator=g) * 0.1
+    w2 = torch.randn(dh, generator=g) * 0.5
+    ref_score = O.mlp_router_score(S.bf16_bits(hid.h), S.bf16_bits(W1), b1.numpy(), w2.numpy(), -0.1)
+    tau = float(np.median(ref_score))
+    near = np.abs(ref_score - tau) <= 1e-3
+    want = O.route_decision(ref_score, tau)[0]
+
+    codes, scale = S.make_W8(d, V, seed=3, std=0.1)
+    r8 = pkg.Router(codes.cuda(), max_n=n, wscale=scale.cuda())
+    r8.set_router_mlp(W1.cuda(), b1.cuda(), w2.cuda(), -0.1)
+    scores = torch.full((n,), float("nan"), device="cuda")
+    r8.route(hid.h.cuda(), tau, score_source=pkg.TLR_SCORE_MLP, mlp_score=scores)
+    torch.cuda.synchronize()
+    assert pkg.tlr_last_device_status(r8.ctx) == 0
+    assert np.max(np.abs(scores.cpu().numpy() - ref_score)) <= 1e-3
+    assert np.array_equal(r8.route_mask[:n].cpu().numpy()[~near], want[~near])
+    r8.close()
+
+    r = pkg.Router(S.make_W(d, V, seed=3, std=0.1).cuda(), max_n=n)
+    r.set_router_mlp(W1.cuda(), b1.cuda(), w2.cuda(), -0.1)
+    assert pkg.tlr_plan_query(r.ctx, n).launches == 2
+    buf = hid.h.cuda().clone()
+    scores.fill_(float("nan"))
+    r.route(buf, tau, score_source=pkg.TLR_SCORE_MLP, mlp_score=scores)          # eager first (one-time set-up)
+    torch.cuda.synchronize()
+    eager = (scores.cpu().numpy().copy(), r.route_mask[:n].cpu().numpy().copy(), int(r.routed_count.item()))
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph, stream=side):
+        r.route(buf, tau, score_source=pkg.TLR_SCORE_MLP, mlp_score=scores)
+    scores.fill_(float("nan")); r.route_mask.fill_(9)
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(scores.cpu().numpy(), eager[0]) and np.array_equal(r.route_mask[:n].cpu().numpy(), eager[1])
+    assert int(r.routed_count.item()) == eager[2]
+    assert np.max(np.abs(eager[0] - ref_score)) <= 1e-3 and np.array_equal(eager[1][~near], want[~near])
+    del graph
+    r.close()
