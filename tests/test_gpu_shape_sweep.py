@@ -2,7 +2,8 @@
 
 The fixed lists of the other parity tests were chosen by hand around the switches of the planner (64 / 128 / 256
 rows, 16 / 32 / 64 rows per part on the 8-bit head, one CTA or a pair per worker, tiles of 16..256 vocabulary
-rows); this file draws shapes nobody chose.  TLR_SWEEP_CASES widens the sweep (default 40 + 16 cases).
+rows); this file draws shapes nobody chose, with and without the learned router.  TLR_SWEEP_CASES widens the sweep
+(default 40 + 16 + 12 cases).
 """
 import os
 
@@ -65,3 +66,51 @@ def test_8bit_head_on_a_drawn_shape(pkg, n, d, V):
     if rep["route_exempt_rows"] == 0:
         assert gpu["routed_count"] == ref.routed_count
         assert np.array_equal(gpu["routed_idx"][:ref.routed_count], ref.routed_idx)
+
+
+def draw_router_shapes(count, seed):
+    rng = np.random.default_rng(seed)
+    shapes = []
+    while len(shapes) < count:
+        n = int(round(np.exp(rng.uniform(np.log(2), np.log(900)))))
+        d = 8 * int(round(np.exp(rng.uniform(np.log(1), np.log(160)))))
+        dh = int(round(np.exp(rng.uniform(np.log(1), np.log(700)))))
+        V = int(round(np.exp(rng.uniform(np.log(2), np.log(60000)))))
+        if n * d * (V + dh) > 1.0e9:
+            continue
+        shapes.append((n, d, dh, V))
+    return shapes
+
+
+@pytest.mark.parametrize("n,d,dh,V", draw_router_shapes(max(1, (CASES * 3) // 10), seed=11))
+def test_learned_router_inside_the_launch_on_a_drawn_shape(pkg, n, d, dh, V):
+    W = S.make_W(d, V, seed=n + V, std=0.1)
+    hid = S.make_h(n, d, seed=n + dh)
+    g = torch.Generator().manual_seed(dh + d)
+    W1 = (torch.randn(dh, d, generator=g) / d ** 0.5).to(torch.bfloat16)
+    b1 = torch.randn(dh, generator=g) * 0.1
+    w2 = torch.randn(dh, generator=g) * 0.5
+    b2 = -0.1
+    ref_score = O.mlp_router_score(S.bf16_bits(hid.h), S.bf16_bits(W1), b1.numpy(), w2.numpy(), b2)
+    base = O.route_oracle(S.bf16_bits(hid.h), S.bf16_bits(W), 0.5)
+    tau = float(np.median(ref_score))
+    want = O.route_decision(ref_score, tau)
+    r = pkg.Router(W.cuda(), max_n=n)
+    r.set_router_mlp(W1.cuda(), b1.cuda(), w2.cuda(), b2)
+    scores = torch.full((n,), float("nan"), device="cuda")
+    r.route(hid.h.cuda(), tau, score_source=pkg.TLR_SCORE_MLP, mlp_score=scores)
+    torch.cuda.synchronize()
+    assert pkg.tlr_last_device_status(r.ctx) == 0
+    got = scores.cpu().numpy()
+    assert np.max(np.abs(got - ref_score)) <= 1e-3
+    mask = r.route_mask[:n].cpu().numpy()
+    near = np.abs(ref_score - tau) <= 1e-3
+    assert np.array_equal(mask[~near], want[0][~near])
+    assert np.array_equal(mask == 1, got < np.float32(tau))
+    c = int(r.routed_count.item())
+    assert c == int(mask.sum()) and np.array_equal(r.routed_idx[:c].cpu().numpy(), np.flatnonzero(mask))
+    sure = base.top2_gap >= 1e-3
+    assert np.array_equal(r.token[:n].cpu().numpy()[sure], base.token[sure])
+    assert np.max(np.abs(r.conf[:n].cpu().numpy() - base.conf) / base.conf) <= 1e-3
+    assert np.max(np.abs(r.entropy[:n].cpu().numpy() - base.entropy)) <= 1e-3
+    r.close()
