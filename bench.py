@@ -137,6 +137,10 @@ def physical_gpu_index(local_rank):
     return local_rank
 
 
+NOMINAL_HBM_GBS = 8000.0        # HBM3e, datasheet
+NOMINAL_BF16_TFLOPS = 2250.0    # dense bf16, datasheet
+
+
 def roofline_fractions(n, d, V, seconds, peaks, fp8=False):
     """The three fractions every record carries, from one duration: HBM, tensor against the burst cuBLAS
     figure, tensor against the sustained one; and the ridge reading max(t_mem, t_mma) / t with t_mma at the
@@ -146,7 +150,10 @@ def roofline_fractions(n, d, V, seconds, peaks, fp8=False):
     t_mma = fl / (float(peaks["bf16_tflops"]) * 1e12)
     t_mma_sus = fl / (float(peaks.get("bf16_tflops_sustained", peaks["bf16_tflops"])) * 1e12)
     return {"hbm_frac": t_mem / seconds, "tensor_frac_burst": t_mma / seconds,
-            "tensor_frac_sustained": t_mma_sus / seconds, "ridge_frac": max(t_mem, t_mma) / seconds}
+            "tensor_frac_sustained": t_mma_sus / seconds, "ridge_frac": max(t_mem, t_mma) / seconds,
+            # the same duration against the datasheet figures (context; the measured peaks are the roofline)
+            "hbm_frac_of_nominal": by / (NOMINAL_HBM_GBS * 1e9) / seconds,
+            "tensor_frac_of_nominal": fl / (NOMINAL_BF16_TFLOPS * 1e12) / seconds}
 
 
 def time_steps(P, routers, step, steps, sampler, world, kernel_steps):

@@ -22,6 +22,9 @@ def test_fractions_follow_from_one_duration_and_the_three_peaks():
     assert f["tensor_frac_sustained"] == pytest.approx(1185.4 / 1385.8, abs=2e-4)
     # ridge reading: the longer of t_mem = 41.70 us and t_mma = 42.75 us over the measured time
     assert f["ridge_frac"] == pytest.approx(42.754 / 58.8, abs=2e-4)
+    # against the datasheet figures (8 TB/s, 2.25 PFLOP/s dense bf16): 4638 / 8000 and 1185.4 / 2250
+    assert f["hbm_frac_of_nominal"] == pytest.approx(0.5798, abs=2e-4)
+    assert f["tensor_frac_of_nominal"] == pytest.approx(0.5268, abs=2e-4)
     # a tensor-bound shape: the HBM fraction is tiny and the ridge reading equals the tensor one
     g = bench.roofline_fractions(8192, 896, 151936, 1.7717e-3, peaks)
     assert g["tensor_frac_sustained"] == pytest.approx(0.908, abs=2e-3) and g["hbm_frac"] < 0.03
