@@ -351,7 +351,7 @@ def run_ours(args):
         tau = args.tau
     fp8 = bool(args.fp8)
     if fp8 and n > 64:
-        raise SystemExit("--fp8 serves decode batches only (n <= 64): pick decode16 or sweep1/8/64")
+        raise SystemExit("--fp8 serves decode batches only (n <= 128): pick decode16 or sweep1/8/64")
     # two device copies of W, alternated step by step: together with W > L2 (or, for the 8-bit copy
     # of the 0.5B head, two copies > L2) this makes every step stream W from HBM rather than from
     # whatever the previous step left in L2
@@ -730,7 +730,7 @@ def main():
                          "(tlr_route_ex; sequences of --seq-len rows)")
     ap.add_argument("--seq-len", type=int, default=0)
     ap.add_argument("--fp8", action="store_true",
-                    help="decode workloads (n <= 64) on an 8-bit copy of W (tlr_create_fp8); the roofline then "
+                    help="decode workloads (n <= 128) on an 8-bit copy of W (tlr_create_fp8); the roofline then "
                          "counts one byte per weight")
     ap.add_argument("--mlp", type=int, default=0,
                     help="attach a learned router of this hidden width (random weights) and route on its score")

@@ -302,13 +302,13 @@ tlr_status tlr_route_host_collect(tlr_ctx* ctx, int32_t* token_host, float* conf
  * 8-bit float: 1 sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, 0x7f / 0xff
  * are NaN), row-major [V, d], 16-byte aligned, and wscale_dev one float per row, so that
  * W[v][k] = wscale[v] * value(code[v][k]).  Both are device memory, BORROWED for the life of the
- * context.  d must be a multiple of 16.  Calls on this context accept n <= 64 rows
+ * context.  d must be a multiple of 16.  Calls on this context accept n <= 128 rows
  * (TLR_ERR_UNSUPPORTED above: larger batches are bound by the tensor cores, not by HBM, and gain
  * nothing from a smaller W); h stays bf16 and is NOT rounded to 8 bits -- each call splits it
  * into two e4m3 parts whose sum is the bf16 value (exact down to 2^-10 of a row's largest
  * element), so the result is that of the bf16 path run on the de-quantised W, to fp32 rounding.
  * All other calls (tlr_route, tlr_route_ex, tlr_route_host, ...) work on the context unchanged;
- * tlr_set_path(TLR_PATH_SIMT) is not available.  Allocates like tlr_create, plus 2 x 64 x d bytes.
+ * tlr_set_path(TLR_PATH_SIMT) is not available.  Allocates like tlr_create, plus 2 x 128 x d bytes.
  */
 tlr_status tlr_create_fp8(int32_t d, int32_t V, const void* W_e4m3_dev, const float* wscale_dev, int32_t max_n,
                           tlr_ctx** out);

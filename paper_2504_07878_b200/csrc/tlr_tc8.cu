@@ -68,10 +68,12 @@ h_split_kernel(const __nv_bfloat16* __restrict__ h, int n, int d, int part_rows,
   }
 }
 
-int tc8_max_rows() { return 64; }
+int tc8_max_rows() { return 128; }
 
 void tc8_configure(int n, int d, TcConfig* c) {
-  int part_rows = n <= 16 ? 16 : (n <= 32 ? 32 : 64);      // per part; the operand slab stacks two parts
+  // rows per part; the operand slab stacks the two parts.  Up to 64 rows both parts go through one MMA (its M holds
+  // 2 x 16, 32 or 64 rows); above, every K step takes two MMAs and a part is n rounded up to 16 rows.
+  int part_rows = n <= 16 ? 16 : (n <= 32 ? 32 : (n <= 64 ? 64 : ((n + 15) / 16) * 16));
   const int a_stage = 2 * part_rows * kRowBytes;
   const int b_stage = kBlockN * kRowBytes;
   const int k_slabs = (d + kRowBytes - 1) / kRowBytes;
@@ -83,7 +85,8 @@ void tc8_configure(int n, int d, TcConfig* c) {
   // ... and only while the resident copy leaves the W ring five stages: with four (d = 2048) what the
   // missing launch gains is lost again to the shallower ring
   if (inl && (budget - k_slabs * a_stage) / b_stage < 5) inl = false;
-  int sa = inl ? k_slabs : (part_rows <= 32 ? 6 : 4);
+  int sa = inl ? k_slabs : (part_rows <= 32 ? 6 : (part_rows <= 64 ? 4 : 3));
+  if (!inl && tuning().ring_a > 0) sa = tuning().ring_a;
   int sb = (budget - sa * a_stage) / b_stage;
   if (sb > kMaxBStages) sb = kMaxBStages;
   c->cta = 1;

@@ -322,6 +322,10 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
   // accumulator row r lives in TMEM lane 32 * (r / 16) + r % 16, i.e. in lanes 0..15 of each 32-lane
   // quadrant (checked on the device), so an epilogue warp then holds 16 rows instead of 32.
   const bool m64 = kCta == 1 && p.a_rows <= 64;
+  // 8-bit head with more than 64 token rows: the two parts of h no longer fit one MMA's M (128 at most with one
+  // CTA), so every K step issues two MMAs -- first parts, then second parts, into the same accumulator rows --
+  // and the epilogue reads finished logits as on the bf16 head (no hand-over between warps).
+  const bool wide = kFp8 && p.part_rows > 64;
   const int k_slabs = (p.d + kSlabElems - 1) / kSlabElems;
   const int units = (p.chunks + (p.mlp_hidden > 0 ? 1 : 0)) * p.row_units;
   const int T = p.tiles_per_unit;
@@ -421,6 +425,7 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
       const uint32_t b_lo0 = desc_lo_fixed | ((b_ring & 0x3ffffu) >> 4);
       const uint32_t a_step = a_stage_bytes >> 4, b_step = b_stage_bytes >> 4;
       const int mma_m = m64 ? 64 : kBlockM * kCta;
+      const uint32_t part_off = static_cast<uint32_t>(p.part_rows * kRowBytes) >> 4;   // second parts, in descriptor units
       if (inl) {                                  // h is resident once the nine warps have split it
         ok = __all_sync(0xffffffffu, mbar_wait(h_ready, 0, abort_flag, p.status, wait_ns));
         tc_fence_after();
@@ -456,9 +461,10 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
 #pragma unroll
               for (int k = 0; k < 4; ++k) {
                 // a quarter of the swizzle span along K (16 bf16 or 32 e4m3) = +32 bytes = +2 in the address field
-                if (kFp8)
+                if (kFp8) {
                   umma_e4m3(d_tmem, desc_hi | (a_lo + 2u * k), desc_hi | (b_lo + 2u * k), idesc, (ks | k) != 0 ? 1u : 0u);
-                else
+                  if (wide) umma_e4m3(d_tmem, desc_hi | (a_lo + part_off + 2u * k), desc_hi | (b_lo + 2u * k), idesc, 1u);
+                } else
                   umma_bf16<kCta>(d_tmem, desc_hi | (a_lo + 2u * k), desc_hi | (b_lo + 2u * k), idesc,
                                   (ks | k) != 0 ? 1u : 0u);
               }
@@ -481,16 +487,18 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
     // different lane quadrants (quadrant q and q + shift), so different warps read them: the warp of the second
     // part (the donor) passes its 32 columns through shared memory to the warp of the first part, which adds
     // them, applies the scales and folds.
-    const int shift = kFp8 ? (p.part_rows == 16 ? 1 : 2) : 4;
-    const bool donor = kFp8 && quad >= shift && quad < 2 * shift;
-    const bool idle = kFp8 && quad >= 2 * shift;                       // quadrants that hold no operand rows
+    const int shift = (kFp8 && !wide) ? (p.part_rows == 16 ? 1 : 2) : 4;
+    const bool donor = kFp8 && !wide && quad >= shift && quad < 2 * shift;
+    const bool idle = kFp8 && !wide && quad >= 2 * shift;              // quadrants that hold no operand rows
     const int cquad = donor ? quad - shift : quad;                     // quadrant of the rows this warp works for
     const int row_in_cta = m64 ? cquad * 16 + (lane & 15) : cquad * 32 + lane;
     const bool lane_has_row = !m64 || lane < 16;   // with M = 64 the upper half of a quadrant holds nothing
     const int hx = grp * 2 + cquad;                // hand-over buffer / scale area of this warp pair
     const int hx_lanes = m64 ? 16 : 32;
     float* hx_buf = hx_area + hx * 32 * hx_lanes;
-    float* ws = scale_area + hx * kBlockN;
+    // (more than 64 rows: all eight warps fold and each stages the tile's scales for itself, in the area the
+    // hand-over buffers do not need then)
+    float* ws = wide ? hx_area + (grp * 4 + quad) * kBlockN : scale_area + hx * kBlockN;
     uint32_t hx_n = 0;                       // hand-overs done so far by this warp
     int acc = 0;
     uint32_t acc_phase = 0;
@@ -545,7 +553,16 @@ __device__ __forceinline__ void tc_projection_body(const TcMaps& maps, const TcP
             __syncwarp();                           // the load below is warp-collective
             tmem_ld32(taddr + c0, z);
             tmem_ld_wait();
-            if (kFp8) {
+            if (kFp8 && wide) {
+#pragma unroll
+              for (int j = 0; j < 32; j += 4) {
+                const float4 w4 = *reinterpret_cast<const float4*>(ws + c0 + j);
+                z[j] = z[j] * hs * w4.x;
+                z[j + 1] = z[j + 1] * hs * w4.y;
+                z[j + 2] = z[j + 2] * hs * w4.z;
+                z[j + 3] = z[j + 3] * hs * w4.w;
+              }
+            } else if (kFp8) {
               if (donor) {
                 // second parts: wait until the partner has taken the previous 32 columns, then hand these over
                 if (hx_n > 0 && !mbar_wait(hx_empty(hx), (hx_n - 1) & 1u, abort_flag, p.status, wait_ns)) { ok = false; break; }

@@ -45,7 +45,7 @@ class VocabShardedRouter:
 
     def __init__(self, W_shard: torch.Tensor, v_offset: int, max_n: int, world: int, group=None, wscale=None):
         """W_shard: this rank's rows of W, bf16 [V_local, d]; or, with wscale (float32 [V_local]), their e4m3 codes
-        (decode batches of up to 64 rows, see tlr_create_fp8)."""
+        (decode batches of up to 128 rows, see tlr_create_fp8)."""
         fp8 = wscale is not None
         ok_dtype = W_shard.dtype in (torch.uint8, torch.float8_e4m3fn) if fp8 else W_shard.dtype == torch.bfloat16
         if not (W_shard.is_cuda and ok_dtype and W_shard.dim() == 2 and W_shard.is_contiguous()):

@@ -61,9 +61,10 @@ def planted_h(n, d, W64, seed):
     return torch.from_numpy(g).to(torch.bfloat16)
 
 
-# several tiles and chunks, ragged vocabulary tails, d not a multiple of the 128-wide slab, 1..64 rows
+# several tiles and chunks, ragged vocabulary tails, d not a multiple of the 128-wide slab, 1..128 rows (above 64
+# rows the two parts of h take an MMA each)
 SHAPES = [(16, 128, 1024), (5, 256, 3000), (64, 896, 20011), (33, 144, 777), (1, 64, 300), (48, 2048, 5000),
-          (17, 16, 40)]
+          (17, 16, 40), (65, 128, 3000), (100, 896, 20011), (128, 2048, 5000), (81, 272, 1500), (128, 64, 70000)]
 
 
 @pytest.mark.parametrize("n,d,V", SHAPES)
@@ -87,13 +88,13 @@ def test_fp8_head_matches_oracle_on_dequantised_matrix(pkg, n, d, V):
 # The shapes the benchmark times with --fp8, in its launch configuration: the 0.5B-class head with 16 rows
 # (the kernel splits h itself) and the d = 2048 head of the batch sweep with 1 and 64 rows (separate split kernel,
 # shallower W ring).  Every row is compared with the oracle on the de-quantised matrix.
-FULL_SIZE = [("decode16", 16, True), ("sweep1", 1, False), ("sweep64", 64, False)]
+# Last: the 0.5B-class head with 128 rows, where every K step takes two MMAs (one per part of h).
+FULL_SIZE = [("decode16", 16, True), ("sweep1", 1, False), ("sweep64", 64, False), ("decode16", 128, False)]
 
 
 @pytest.mark.parametrize("name,n,inline", FULL_SIZE)
 def test_fp8_head_at_benchmark_sizes(pkg, name, n, inline):
     wl = S.WORKLOADS[name]
-    assert wl.n == n
     codes, scale = FullHead8.get(wl.d, wl.V)
     W64 = FullHead8.w64
     hid = S.make_h(n, wl.d, seed=0)
@@ -164,11 +165,11 @@ def test_fp8_argument_errors(pkg):
     assert L.tlr_create_fp8(64, 500, P(cd.data_ptr()), P(0), 8, ctypes.byref(ctx)) == 1          # no scales
     assert L.tlr_create_fp8(64, 500, P(cd.data_ptr() + 1), P(sd.data_ptr()), 8, ctypes.byref(ctx)) == 2
     assert L.tlr_create_fp8(72, 400, P(cd.data_ptr()), P(sd.data_ptr()), 8, ctypes.byref(ctx)) == 3   # d % 16 != 0
-    r = pkg.Router(cd, max_n=100, wscale=sd)
-    h = torch.zeros((65, 64), dtype=torch.bfloat16, device="cuda")
+    r = pkg.Router(cd, max_n=200, wscale=sd)
+    h = torch.zeros((129, 64), dtype=torch.bfloat16, device="cuda")
     with pytest.raises(pkg.TlrError) as e:
         r.route(h, 0.5)
-    assert e.value.code == 3                                                                         # more than 64 rows
+    assert e.value.code == 3                                                                         # more than 128 rows
     with pytest.raises(pkg.TlrError):
         pkg.tlr_set_path(r.ctx, pkg.TLR_PATH_SIMT)
     r.close()

@@ -51,7 +51,7 @@ def test_bf16_head_on_a_drawn_shape(pkg, n, d, V):
         assert np.array_equal(gpu["routed_idx"][:ref.routed_count], ref.routed_idx)
 
 
-@pytest.mark.parametrize("n,d,V", draw_shapes(max(1, (CASES * 2) // 5), seed=77, n_max=64, d_step=16))
+@pytest.mark.parametrize("n,d,V", draw_shapes(max(1, (CASES * 2) // 5), seed=77, n_max=128, d_step=16))
 def test_8bit_head_on_a_drawn_shape(pkg, n, d, V):
     codes, scale = S.make_W8(d, V, seed=n + d + V, std=0.1)
     W64 = O.dequantize_e4m3(codes.numpy(), scale.numpy())
