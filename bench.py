@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc_kernel.cuh", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
-    "sha256": "8f981209b227a46ae19d6a61e9ebc657ce578214267aa60cccf3d27c1aaf28d7",
-    "bytes_per_launch": {"decode256": 277.65e6, "decode16": 276.39e6, "sweep512": 532.87e6},
+    "sha256": "0b2c6fb0392d1bc87b171e79cb99aa84f105fd5f28dc72f0d9ed10097998538d",
+    "bytes_per_launch": {"decode256": 274.44e6, "decode16": 274.32e6, "sweep512": 529.54e6},
 }
 
 
