@@ -350,8 +350,8 @@ def run_ours(args):
     if args.tau is not None:
         tau = args.tau
     fp8 = bool(args.fp8)
-    if fp8 and n > 64:
-        raise SystemExit("--fp8 serves decode batches only (n <= 128): pick decode16 or sweep1/8/64")
+    if fp8 and n > 128:
+        raise SystemExit("--fp8 serves decode batches only (n <= 128): pick decode16 or sweep1/8/64, or --rows N")
     # two device copies of W, alternated step by step: together with W > L2 (or, for the 8-bit copy
     # of the 0.5B head, two copies > L2) this makes every step stream W from HBM rather than from
     # whatever the previous step left in L2
@@ -505,7 +505,7 @@ def run_ours(args):
         achieved = algorithmic_flops(n, d, V) / (kernel_ms * 1e-3) / 1e12
         roof = {"bound": "tensor", "achieved": achieved, "peak": float(peaks["bf16_tflops"]), "unit": "TFLOP/s",
                 "frac": kfr["tensor_frac_burst"], "peak_kind": "burst"}
-    roof.update({"traffic": None if fp8 else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
+    roof.update({"traffic": None if (fp8 or args.rows > 0) else ncu_traffic(wl.name), "algorithmic_bytes": algorithmic_bytes(n, d, V, fp8),
                  "algorithmic_flops": algorithmic_flops(n, d, V), "peak_source": "of " + peak_kind,
                  "kernel": ("h_split_kernel + tc8_projection_kernel" if fp8 else
                             "tc_projection_kernel" if plan.path == P.TLR_PATH_TC else "simt_projection_kernel"),
@@ -737,9 +737,15 @@ def main():
     ap.add_argument("--one-shard-of", type=int, default=0, metavar="G",
                     help="one GPU: time the work of ONE rank of a G-way vocabulary-sharded step (fused exchange), "
                          "a decode workload's batch on V / G rows of W")
+    ap.add_argument("--rows", type=int, default=0, metavar="N",
+                    help="time the workload's head with a batch of N rows instead of its own (the line's "
+                         "config.workload says so)")
     args = ap.parse_args()
     if args.warmup < 3:
         args.warmup = 3
+    if args.rows > 0:
+        import dataclasses
+        S.WORKLOADS[args.workload] = dataclasses.replace(S.WORKLOADS[args.workload], n=args.rows)
     if args.impl == "torch-eager":
         run_torch_eager(args)
     elif args.impl == "reference":
