@@ -36,8 +36,8 @@ RIDGE_ROWS_HBM = 256            # at or below this many rows the step is reporte
 # hash of that source is recorded here and traffic is reported as null when the source differs.
 NCU_TRAFFIC = {
     "kernel_sources": ["paper_2504_07878_b200/csrc/tlr_tc_kernel.cuh", "paper_2504_07878_b200/csrc/tlr_tc_ptx.cuh"],
-    "sha256": "0b2c6fb0392d1bc87b171e79cb99aa84f105fd5f28dc72f0d9ed10097998538d",
-    "bytes_per_launch": {"decode256": 274.44e6, "decode16": 274.32e6, "sweep512": 529.54e6},
+    "sha256": "ad20ef2b7c5159246522e6c7c2b720eb8a483e50cce12ecae6fcb02813170e00",
+    "bytes_per_launch": {"decode256": 274.54e6, "decode16": 274.09e6, "sweep512": 529.42e6},
 }
 
 

@@ -9,10 +9,11 @@
 //               CTA stages its own 128 rows of h and HALF of the W tile, and the pair's
 //               tensor cores read both halves, so a W byte enters shared memory once
 //               per 256 token rows.                                       (n > 128)
-//   <1, true>   8-bit (e4m3) head for decode batches of at most 64 rows: h is the sum of two e4m3
-//               parts, stacked along M in one operand slab (rows 0.. = first parts, rows
-//               part_rows.. = second parts), ONE kind::f8f6f4 MMA per K step; the epilogue adds
-//               the two accumulator rows of a token before it folds them.
+//   <1, true>   8-bit (e4m3) head for decode batches of at most 128 rows: h is the sum of two e4m3
+//               parts, stacked in one operand slab (rows 0.. = first parts, rows part_rows.. =
+//               second parts).  Up to 64 rows ONE kind::f8f6f4 MMA per K step covers both parts
+//               along its M, and the epilogue adds the two accumulator rows of a token before it
+//               folds them; above, two MMAs per K step (one per part) add into the same rows.
 //
 // Decomposition.  The vocabulary is cut into `chunks` contiguous ranges of granules
 // (a multiple of 16 * kCta rows); the token rows into units of 128 * kCta.  A work unit is
@@ -80,6 +81,7 @@ constexpr int kSmemLimit = 232448;           // 227 KiB opt-in maximum per CTA
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;  // 2 s
 // 8-bit head: weight scales of a tile for each of the four warps that fold, the rows' power-of-two scales,
 // and four hand-over buffers (32 columns x lanes floats) between the warps that hold a token's two parts
+// (with more than 64 rows nothing is handed over and the buffers' space holds the scales for all eight warps)
 constexpr int kScaleBytes = 4 * kBlockN * 4;
 constexpr int kRowScaleBytes = 64 * 4;
 __host__ __device__ constexpr int tc8_extra_bytes(int part_rows) {
