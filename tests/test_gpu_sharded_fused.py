@@ -166,3 +166,38 @@ def test_row_sharded_lists_merge_into_the_global_list(pkg, rows_per_rank, d, V):
     router.close()
     with pytest.raises(pkg.TlrError):
         pkg.tlr_rows_merge(gathered, counts, None, world, cap, out, n_out)
+
+
+@pytest.mark.parametrize("n", [24, 100])        # one MMA per K step / one per part of h
+def test_fused_exchange_on_the_8bit_head(pkg, n):
+    """Shards of an e4m3 head (codes and scales cut at the same rows) with the exchange fused into the kernels,
+    against the oracle on the de-quantised matrix."""
+    d, V, shards = 128, 9000, 4
+    codes, scale = S.make_W8(d, V, seed=8, std=0.1)
+    W64 = O.dequantize_e4m3(codes.numpy(), scale.numpy())
+    h = S.make_h(n, d, seed=n).h
+    first = O.route_oracle(S.bf16_bits(h), None, 0.5, W64=W64)
+    tau = O.percentile_tau(first.conf, 0.5)
+    ref = O.with_threshold(first, tau)
+    cd, sd, hd = codes.cuda(), scale.cuda(), h.cuda()
+    block = torch.zeros(pkg.tlr_shard_block_bytes(n, shards), dtype=torch.uint8, device="cuda")
+    ranks = []
+    for g in range(shards):
+        v0, v1 = pkg.shard_bounds(V, shards, g)
+        ranks.append(pkg.FusedVocabShardedRouter(cd[v0:v1], v0, n, g, shards, [block] * shards, wscale=sd[v0:v1],
+                                                 keep=block))
+    for r in ranks:
+        r.push(hd)
+    poison(ranks[2])
+    ranks[2].finish(n, tau)
+    torch.cuda.synchronize()
+    for r in ranks:
+        assert pkg.tlr_last_device_status(r.ctx) == 0
+    gpu = outputs(ranks[2], n)
+    check_self_consistency(gpu, tau, V)
+    rep = check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(h)), W64)
+    if rep["route_exempt_rows"] == 0:
+        assert gpu["routed_count"] == ref.routed_count
+        assert np.array_equal(gpu["routed_idx"][:ref.routed_count], ref.routed_idx)
+    for r in ranks:
+        r.close()
