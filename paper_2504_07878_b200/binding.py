@@ -350,6 +350,24 @@ class Router:
         return (self.token[:n], self.conf[:n], self.entropy[:n], self.route_mask[:n], self.routed_idx,
                 self.routed_count)
 
+    def prepared(self, h: torch.Tensor, tau: float, stream=None):
+        """The same step as route(h, tau, stream) as a callable with its arguments marshalled once: for a decode
+        loop that calls again and again with the same buffers, each call is then a single foreign call.  The
+        outputs are this router's tensors, as with route()."""
+        if not (h.is_cuda and h.dtype == torch.bfloat16 and h.dim() == 2 and h.is_contiguous()
+                and h.shape[1] == self.d):
+            raise ValueError("h must be a contiguous CUDA bf16 [n, d] tensor")
+        fn = load_library().tlr_route
+        args = (self.ctx, _ptr(h), int(h.shape[0]), float(tau), _ptr(self.token), _ptr(self.conf), _ptr(self.entropy),
+                _ptr(self.route_mask), _ptr(self.routed_idx), _ptr(self.routed_count), _stream_handle(stream))
+        keep = (h, stream, self)       # the buffers stay alive as long as the callable does
+
+        def call():
+            _check(fn(*args), "tlr_route")
+            return keep[2]
+
+        return call
+
     def close(self):
         if self.ctx is not None:
             tlr_destroy(self.ctx)

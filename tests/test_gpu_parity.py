@@ -292,3 +292,25 @@ def test_degenerate_vocabulary_and_tiny_shapes(pkg, path):
         assert gpu["status"] == 0
         check_self_consistency(gpu, 0.3, V)
         check_against_oracle(ref, gpu, O.bf16_bits_to_f64(S.bf16_bits(hid.h)), O.bf16_bits_to_f64(S.bf16_bits(W)))
+
+
+def test_prepared_call_is_the_same_step(pkg):
+    """Router.prepared marshals the arguments once; calling it is bit-identical to route()."""
+    W, hid = small_case(150, 128, 6000, seed=21, planted=0.1)
+    r = pkg.Router(W.cuda(), max_n=150)
+    h = hid.h.cuda()
+    r.route(h, 0.4)
+    torch.cuda.synchronize()
+    want = [t.clone() for t in (r.token, r.conf, r.entropy, r.route_mask, r.routed_count)]
+    want_idx = r.routed_idx[:int(r.routed_count.item())].clone()
+    call = r.prepared(h, 0.4)
+    for _ in range(3):
+        r.token.fill_(-1); r.routed_count.fill_(-1)
+        call()
+    torch.cuda.synchronize()
+    for got, w in zip((r.token, r.conf, r.entropy, r.route_mask, r.routed_count), want):
+        assert torch.equal(got, w)
+    assert torch.equal(r.routed_idx[:int(r.routed_count.item())], want_idx)
+    with pytest.raises(ValueError):
+        r.prepared(h.float(), 0.4)
+    r.close()
