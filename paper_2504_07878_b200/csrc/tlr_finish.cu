@@ -9,8 +9,9 @@
 //
 // Compaction (ballot / popcount / prefix sum, ascending order):
 //   n <= 1024  a thread-block cluster of up to 8 blocks folds the rows (a group of L lanes
-//              per row, all rows at once); after a cluster barrier block 0 compacts the
-//              flags.  No ticket, no second launch, about two L2 round trips.  The blocks
+//              per row, all rows at once) and store the route flags into block 0's shared memory;
+//              after a cluster barrier block 0 compacts them.  No ticket, no second launch, one L2
+//              round trip for the partials.  The blocks
 //              have 512 threads where a lane group still owns at most 6 partials (else 1024):
 //              that size fits on an SM beside a CTA of the tensor-core projection kernel, so
 //              the blocks are resident and waiting before that kernel ends, and the next
@@ -267,14 +268,23 @@ finish_small_kernel(const FinishLaunch a, const int L) {
       acc.s = s;
       acc.t = t;
       const int f = score_row(acc, a, row);
-      if (single_block) flags[row] = static_cast<unsigned char>(f);
+      if (single_block) {
+        flags[row] = static_cast<unsigned char>(f);
+      } else {
+        // into block 0's shared memory (distributed shared memory of the cluster): block 0 then compacts
+        // without another trip to L2 for the flags
+        const uint32_t mine = static_cast<uint32_t>(__cvta_generic_to_shared(&flags[row]));
+        uint32_t remote;
+        asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(remote) : "r"(mine), "r"(0));
+        asm volatile("st.shared::cluster.u8 [%0], %1;" ::"r"(remote), "r"(f) : "memory");
+      }
     }
   }
   if (single_block) {
     __syncthreads();                    // the flags are in this block's shared memory
   } else {
-    // Every block's flags are in route_mask; the cluster barrier (release / acquire) makes
-    // them visible to block 0, which compacts them.
+    // The cluster barrier (release / acquire) makes every block's stores into block 0's shared memory
+    // visible to block 0, and keeps block 0 (and its shared memory) there until they have been made.
     asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
     asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
   }
@@ -285,7 +295,7 @@ finish_small_kernel(const FinishLaunch a, const int L) {
   for (int base = 0; base < a.n; base += blockDim.x) {       // one pass when the block has a thread per row
     const int i = base + threadIdx.x;
     int flag = 0;
-    if (i < a.n) flag = single_block ? static_cast<int>(flags[i]) : static_cast<int>(__ldcg(a.route_mask + i));
+    if (i < a.n) flag = static_cast<int>(flags[i]);
     const unsigned int bal = __ballot_sync(0xffffffffu, flag != 0);
     if (lane == 0) warp_count[warp] = __popc(bal);
     __syncthreads();
