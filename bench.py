@@ -230,8 +230,9 @@ def side_record(P, name, routers, h_dev, tau, seconds, gpu_index, peaks, fp8=Fal
 
 def run_one_rank_of_a_vocab_shard(args):
     """--one-shard-of G on one GPU: the work ONE rank of a G-way vocabulary-sharded step does per call -- the
-    projection over V / G rows of W, the per-row summaries stored into the exchange block (here: its own, the
-    other ranks' slots filled once beforehand), the bounded wait on the flags and the merge.  No exchange
+    projection over V / G rows of W, the per-row summaries stored into the exchange block, the bounded wait on
+    the flags and the merge.  All G ranks run one after the other in one stream (every "peer" block is the same
+    local block): G pushes, then G merges, and the time per rank is that of the loop divided by G.  No exchange
     latency is in it (there is one GPU); it gives the per-rank time a G-GPU run could approach."""
     import paper_2504_07878_b200 as P
     from paper_2504_07878_b200 import build
@@ -244,76 +245,57 @@ def run_one_rank_of_a_vocab_shard(args):
     wl = S.WORKLOADS[args.workload]
     n, d, V = wl.n, wl.d, wl.V
     tau = 0.5 if wl.tau is None else wl.tau
-    W = S.make_W(d, V, seed=0).cuda()
     h = S.make_h(n, d, seed=0).h.cuda()
-    copies = max(2, min(64, int(300e6 // (2 * d * V // G)) + 1))       # enough copies of the shard to exceed L2
-    block = torch.zeros(P.tlr_shard_block_bytes(n, G), dtype=torch.uint8, device="cuda")
-    ranks = []
-    for g in range(G):
-        v0, v1 = P.shard_bounds(V, G, g)
-        ranks.append(P.FusedVocabShardedRouter(W[v0:v1], v0, n, g, G, [block] * G, keep=block))
-    v0, v1 = P.shard_bounds(V, G, 0)
-    mine = [ranks[0]] + [P.FusedVocabShardedRouter(W[v0:v1].clone(), v0, n, 0, G, [block] * G, keep=block)
-                         for _ in range(copies - 1)]
+    # Two complete sets of ranks (each set: the G shards of its own copy of W, its own exchange block) alternate
+    # between steps, so that a step streams its shards from HBM rather than from what the last step left in L2.
+    sets = []
+    W_host = S.make_W(d, V, seed=0)
+    for _ in range(2):
+        W = W_host.cuda()
+        block = torch.zeros(P.tlr_shard_block_bytes(n, G), dtype=torch.uint8, device="cuda")
+        ranks = []
+        for g in range(G):
+            v0, v1 = P.shard_bounds(V, G, g)
+            ranks.append(P.FusedVocabShardedRouter(W[v0:v1], v0, n, g, G, [block] * G, keep=(block, W)))
+        sets.append(ranks)
     stream = torch.cuda.current_stream()
 
-    def others(i):
-        # the other ranks push first, so their summaries for this call number are in the block; the copies of
-        # rank 0 that are not used in this call push an empty batch, which keeps every call counter in step
-        for r in ranks[1:]:
+    def step(i):
+        ranks = sets[i & 1]
+        for r in ranks:
             r.push(h)
-        for c in mine:
-            if c is not mine[i % copies]:
-                P.tlr_shard_push(c.ctx, h[:0], 0, c.v_offset)
-
-    def rank0(i):
-        mine[i % copies].push(h)
-        mine[i % copies].finish(n, tau)
-
-    def timed(loop_body, steps):
-        torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for i in range(steps):
-            loop_body(i)
-        e1.record(stream)
-        torch.cuda.synchronize()
-        return e0.elapsed_time(e1) / steps
-
-    def everything(i):
-        others(i)
-        rank0(i)
+        for r in ranks:
+            r.finish(n, tau)
 
     for i in range(max(3, args.warmup)):
-        everything(i)
+        step(i)
     steps = min(args.steps, 2000)
-    # Back to back in one stream: all ranks' work, and the same loop with rank 0's finish left out but its
-    # push replaced by an empty one (the flags must still be set for the next call); the difference is rank 0's
-    # projection + summaries + merge.
-    ms_all = timed(everything, steps)
-
-    def without_rank0(i):
-        others(i)
-        P.tlr_shard_push(mine[i % copies].ctx, h[:0], 0, mine[i % copies].v_offset)
-
-    ms_rest = timed(without_rank0, steps)
-    ms = ms_all - ms_rest
-    status = max(P.tlr_last_device_status(r.ctx) for r in ranks + mine[1:])
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for i in range(steps):
+        step(i)
+    e1.record(stream)
+    torch.cuda.synchronize()
+    ms_all = e0.elapsed_time(e1) / steps
+    ms = ms_all / G
+    status = max(P.tlr_last_device_status(r.ctx) for ranks in sets for r in ranks)
     if status & P.TLR_DEV_WAIT_TIMEOUT:
         raise SystemExit("device status flags raised: %d" % status)
     peaks, peak_kind = measured_peaks()
+    v0, v1 = P.shard_bounds(V, G, 0)
     shard_bytes = 2 * (v1 - v0) * d + 2 * n * d + 17 * n + 4 + 16 * n * G
     print(json.dumps({"metric": METRIC, "value": n / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
                       "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
                       "vs_baseline": None, "dtype": "bf16 in, fp32 accumulate and softmax statistics", "data": "synthetic",
                       "config": {"workload": "%s, ONE rank's share of a %d-way vocabulary-sharded step: n=%d rows, d=%d, "
                                              "%d of V=%d rows of W, tau=%g" % (wl.name, G, n, d, v1 - v0, V, tau),
-                                 "l2": "%d copies of the shard alternate (together larger than L2); time = a back-to-back loop over "
-                                       "all ranks' calls minus the same loop without rank 0's projection and merge "
-                                       "(%.4f - %.4f ms)" % (copies, ms_all, ms_rest),
+                                 "l2": "two sets of %d ranks (two copies of W) alternate between steps; time = a back-to-back "
+                                       "loop in which all %d ranks push and then all merge (%.4f ms), divided by %d"
+                                       % (G, G, ms_all, G),
                                  "exchange": "fused: summaries stored into the exchange block, flags, bounded wait in "
                                              "the merge kernel (one GPU: no link latency in this number)"},
-                      "gpu_launches": 3 * steps,
+                      "gpu_launches": 3 * G * steps,
                       "roofline": {"bound": "hbm", "achieved": shard_bytes / (ms * 1e-3) / 1e9, "peak": float(peaks["hbm_gbs"]),
                                    "unit": "GB/s", "frac": shard_bytes / (ms * 1e-3) / 1e9 / float(peaks["hbm_gbs"]),
                                    "traffic": None, "algorithmic_bytes": shard_bytes, "peak_source": "of " + peak_kind,

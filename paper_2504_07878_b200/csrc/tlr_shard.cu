@@ -56,6 +56,10 @@ __global__ void __launch_bounds__(kWarps * 32)
 shard_push_kernel(const ShardPush a) {
   const int row = blockIdx.x * kWarps + (threadIdx.x >> 5);
   const int lane = threadIdx.x & 31;
+  // Programmatic dependent launch: scheduled while the projection kernel finishes, and the merge kernel behind
+  // this one may be scheduled now; the partials are read only after the projection has completed.
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+  asm volatile("griddepcontrol.wait;" ::: "memory");
   if (row < a.n) {
     const Partial acc = row_summary(a.partials, row, a.chunks, a.v_offset, lane);
     for (int g = lane; g < a.shards; g += 32) a.peer_slot[g][row] = acc;     // lane g stores to peer g
@@ -108,8 +112,16 @@ cudaError_t launch_shard_summary(const Partial* partials, int n, int chunks, int
 
 cudaError_t launch_shard_push(const ShardPush& a, cudaStream_t stream) {
   const int blocks = a.n > 0 ? (a.n + kWarps - 1) / kWarps : 1;   // n == 0 still publishes the flags
-  shard_push_kernel<<<blocks, kWarps * 32, 0, stream>>>(a);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(blocks), 1, 1);
+  cfg.blockDim = dim3(kWarps * 32, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, shard_push_kernel, a);
 }
 
 cudaError_t launch_rows_merge(const int32_t* gathered_idx, const int32_t* counts, const int32_t* row_offsets,
