@@ -476,8 +476,12 @@ def run_ours(args):
     # ---- N > 1: the vocabulary-sharded form of the same decode batch (one exchange step per call)
     vocab_sharded = None
     if world > 1 and n <= 1024 and not fp8 and not variant_args:
-        vocab_sharded = vocab_sharded_record(P, W_host, S.make_h(n, d, seed=0).h, tau, rank, world, args.steps,
-                                             max(args.warmup, 3))
+        # (a sub-record beside the line's own numbers: an error in it is reported, not allowed to lose the line)
+        try:
+            vocab_sharded = vocab_sharded_record(P, W_host, S.make_h(n, d, seed=0).h, tau, rank, world, args.steps,
+                                                 max(args.warmup, 3))
+        except Exception as e:      # noqa: BLE001
+            vocab_sharded = {"unavailable": "%s: %s" % (type(e).__name__, e)}
 
     if rank != 0:
         return
