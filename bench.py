@@ -472,6 +472,22 @@ def run_ours(args):
         for r in r8:
             r.close()
         del r8, W8
+        # the two other heads of the target (1.5B-class head; the d = 2048 sweep at an HBM-bound and a
+        # tensor-bound batch size): one device copy each, W alone is three to four times L2
+        for names in (("head1p5b",), ("sweep64", "sweep4096")):
+            wlx = S.WORKLOADS[names[0]]
+            Wx = S.make_W(wlx.d, wlx.V, seed=0).cuda()
+            for name in names:
+                wly = S.WORKLOADS[name]
+                rx = [P.Router(Wx, max_n=wly.n)]
+                hx = S.make_h(wly.n, wly.d, seed=0).h.cuda()
+                rec = side_record(P, name, rx, hx, 0.5 if wly.tau is None else wly.tau,
+                                  0.3 if wly.n <= RIDGE_ROWS_HBM else 1.0, gpu_index, peaks)
+                rec["l2"] = "one device copy of W (%.0f MB, larger than L2)" % (2 * wly.V * wly.d / 1e6)
+                also.append(rec)
+                rx[0].close()
+                del rx, hx
+            del Wx
 
     # ---- N > 1: the vocabulary-sharded form of the same decode batch (one exchange step per call)
     vocab_sharded = None
