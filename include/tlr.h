@@ -284,8 +284,10 @@ tlr_status tlr_route_host(tlr_ctx* ctx, const void* h_bf16_host, int32_t n, floa
  * states over PCIe, the kernels' launch and the wake-up of the host overlap the previous batch's kernels
  * (a serving loop that decodes for many sessions has the next batch ready before the last one is back).
  *   submit   enqueues the copy of h to the device, the routing step and the write-back of its results into a
- *            pinned block of the context, and returns without waiting.  h_bf16_host must stay valid and
- *            unchanged until the matching collect has returned.  At most two submitted calls may be waiting to
+ *            pinned block of the context, and returns without waiting.  h_bf16_host must hold the batch when
+ *            submit is called (the GPU may start reading it while earlier work in the stream is still running;
+ *            that work must therefore not be what produces it) and must stay valid and unchanged until the
+ *            matching collect has returned.  At most two submitted calls may be waiting to
  *            be collected (a third returns TLR_ERR_ARG); all on one stream, or on streams the caller orders.
  *   collect  waits for the OLDEST submitted call and hands out its results exactly as tlr_route_host does
  *            (same optional pointers, same TLR_ERR_DEVICE_STATUS rule); TLR_ERR_ARG if none is waiting.

@@ -40,9 +40,19 @@ host_copy_kernel(const uint4* __restrict__ src, uint4* __restrict__ dst, size_t 
 cudaError_t launch_host_copy(const void* src_mapped, void* dst, size_t bytes, cudaStream_t stream) {
   if (bytes == 0) return cudaSuccess;
   if ((bytes & 15u) != 0) return cudaErrorInvalidValue;
-  host_copy_kernel<<<kCopyBlocks, kCopyThreads, 0, stream>>>(static_cast<const uint4*>(src_mapped),
-                                                              static_cast<uint4*>(dst), bytes / 16);
-  return cudaGetLastError();
+  // A programmatic dependent launch itself: the blocks may become resident, and copy, while the kernels of the
+  // previous call in the stream are still running (the wait at the end of the kernel keeps the order of completion).
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(kCopyBlocks, 1, 1);
+  cfg.blockDim = dim3(kCopyThreads, 1, 1);
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, host_copy_kernel, static_cast<const uint4*>(src_mapped), static_cast<uint4*>(dst),
+                            static_cast<size_t>(bytes / 16));
 }
 
 }  // namespace tlr
