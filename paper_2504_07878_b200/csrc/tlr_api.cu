@@ -32,6 +32,7 @@ const Tuning& tuning() {
     }
     if (const char* e = getenv("TLR_TC8_INLINE")) v.tc8_inline = e[0] == '0' ? 0 : 1;
     if (const char* e = getenv("TLR_FINISH_THREADS")) v.finish_threads = atoi(e);
+    if (getenv("TLR_TC_ROW_COST") != nullptr) v.row_cost = 1;
     return v;
   }();
   return t;
@@ -55,7 +56,7 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, int mlp_hidden,
   const long long mlp_cost = mlp_rows + 24 * mlp_tiles;
   int hi = granules < max_chunks ? granules : max_chunks;
   if (hi < 1) hi = 1;
-  long long best_cost = -1;
+  long long best_cost = -1, best_passes = 0;
   int best = 1, best_tiles = 1;
   for (int c = 1; c <= hi; ++c) {
     const long long gmax = (granules + c - 1) / c;
@@ -78,8 +79,15 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, int mlp_hidden,
         if (load > cost) cost = load;
       }
     }
-    if (best_cost < 0 || cost < best_cost) {
+    // Pair mode: a tile costs a pass over all of h whatever its width (the pair MMA takes as long with 32
+    // columns as with 256), so the busiest worker's TILE count is compared first and the row-based cost only
+    // decides between plans with the same count.
+    long long passes = 0;
+    if (cta == 2 && !tuning().even_tiles && !tuning().row_cost && mlp_rows == 0)
+      passes = ((units + workers - 1) / workers) * tiles;
+    if (best_cost < 0 || passes < best_passes || (passes == best_passes && cost < best_cost)) {
       best_cost = cost;
+      best_passes = passes;
       best = c;
       best_tiles = static_cast<int>(tiles);
     }

@@ -84,6 +84,7 @@ struct Tuning {
   int ring_a, ring_b;   // TLR_TC_RINGS="a,b": ring depths (0 = default)
   int tc8_inline;       // TLR_TC8_INLINE=0 keeps the separate split kernel
   int finish_threads;   // TLR_FINISH_THREADS: block size of the merge kernel for n <= 1024 (0 = default)
+  int row_cost;         // TLR_TC_ROW_COST: pair mode plans by vocabulary rows per worker only, not by tile passes first
 };
 const Tuning& tuning();
 

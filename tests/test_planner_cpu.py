@@ -101,3 +101,16 @@ def test_learned_router_costs_the_decode_plans_little():
         a = np.bincount(plain[:, 0], weights=plain[:, 4]).max()
         b = np.bincount(fused[:, 0], weights=fused[:, 4]).max()
         assert b <= 1.03 * a
+
+
+@pytest.mark.parametrize("n,V", [(256, 151936), (512, 128256), (1024, 151936), (4096, 151936), (8192, 151936),
+                                 (4096, 128256), (16384, 128256)])
+def test_pair_mode_minimises_the_busiest_workers_tile_passes(n, V):
+    """With a CTA pair per worker a tile costs a pass over h whatever its width, so the plan must give the busiest
+    worker as few tiles as any chunk count (up to the 192 partials a row may have) allows."""
+    tiles, plan = P.tlr_debug_plan_tiles(n, V, 148)
+    workers, g = plan.grid // 2, plan.reserved
+    busiest = np.bincount(tiles[:, 0]).max()
+    row_units, granules = -(-n // 256), -(-V // g)
+    fewest = min(-(-row_units * c // 74) * -(-(-(-granules // c) * g) // 256) for c in range(1, 193))
+    assert workers <= 74 and busiest == fewest
