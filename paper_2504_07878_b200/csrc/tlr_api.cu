@@ -63,10 +63,15 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, int mlp_hidden,
     const long long tiles = (gmax * g + 255) / 256;
     const long long units = 1ll * row_units * c;
     const long long unit_cost = gmax * g + 24 * tiles;
-    long long cost;
+    // Pair mode: a tile costs a pass over all of h whatever its width (the pair MMA takes as long with 32
+    // columns as with 256), so the busiest worker's TILE count is compared first and the row-based cost only
+    // decides between plans with the same count.
+    const bool by_passes = cta == 2 && !tuning().even_tiles && !tuning().row_cost;
+    long long cost, passes = 0;
     if (mlp_rows == 0) {
       const long long waves = (units + workers - 1) / workers;
       cost = waves * unit_cost;
+      passes = waves * tiles;
     } else {
       // worker w takes units w, w + workers, ...: vocabulary units first, then the row_units router units
       const long long full = units / workers, rem = units % workers;
@@ -77,14 +82,10 @@ void tc_plan(int n, int V, int cta, int workers, int max_chunks, int mlp_hidden,
         const long long nm = j0 < row_units ? 1 + (row_units - 1 - j0) / workers : 0;
         const long long load = nv * unit_cost + nm * mlp_cost;
         if (load > cost) cost = load;
+        if (nv * tiles + nm * mlp_tiles > passes) passes = nv * tiles + nm * mlp_tiles;
       }
     }
-    // Pair mode: a tile costs a pass over all of h whatever its width (the pair MMA takes as long with 32
-    // columns as with 256), so the busiest worker's TILE count is compared first and the row-based cost only
-    // decides between plans with the same count.
-    long long passes = 0;
-    if (cta == 2 && !tuning().even_tiles && !tuning().row_cost && mlp_rows == 0)
-      passes = ((units + workers - 1) / workers) * tiles;
+    if (!by_passes) passes = 0;
     if (best_cost < 0 || passes < best_passes || (passes == best_passes && cost < best_cost)) {
       best_cost = cost;
       best_passes = passes;
