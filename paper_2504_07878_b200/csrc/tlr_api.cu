@@ -145,6 +145,8 @@ struct tlr_ctx {
   unsigned char* out_pinned[2] = {nullptr, nullptr};   // pinned host mirror of the same size, + an aligned 4-byte status word
   unsigned char* out_mapped[2] = {nullptr, nullptr};   // the mirror as the device sees it (kernels write the results into it), or null
   cudaEvent_t slot_done[2] = {nullptr, nullptr};       // recorded behind a submitted call's last kernel
+  cudaStream_t copy_stream = nullptr;                  // large pinned h: copy-engine transfer beside the previous call's kernels
+  cudaEvent_t copy_done[2] = {nullptr, nullptr};       // ... and the event the call's own stream waits for
   int slot_n[2] = {0, 0};
   int slot_next = 0;        // slot of the next submit
   int slots_in_flight = 0;  // submitted and not yet collected (0..2); the oldest is slot (slot_next - in_flight) & 1
@@ -333,7 +335,9 @@ void free_all(tlr_ctx* c) {
     cudaFree(c->out_stage[q]);
     cudaFreeHost(c->out_pinned[q]);
     if (c->slot_done[q] != nullptr) cudaEventDestroy(c->slot_done[q]);
+    if (c->copy_done[q] != nullptr) cudaEventDestroy(c->copy_done[q]);
   }
+  if (c->copy_stream != nullptr) cudaStreamDestroy(c->copy_stream);
   cudaFree(c->mlp_scores);
   cudaFree(c->h_parts);
   cudaFree(c->hscale);
@@ -372,7 +376,9 @@ tlr_status new_context(int d, int V, const void* W_dev, int max_n, tlr_ctx** out
     ok = ok && cudaMalloc(&c->out_stage[q], np * 17 + 8) == cudaSuccess;
     ok = ok && cudaHostAlloc(reinterpret_cast<void**>(&c->out_pinned[q]), np * 17 + 8 + 8, cudaHostAllocMapped) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->slot_done[q], cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->copy_done[q], cudaEventDisableTiming) == cudaSuccess;
   }
+  ok = ok && cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
   if (!ok) {
     cudaGetLastError();
     free_all(c);
@@ -946,13 +952,25 @@ tlr_status tlr_route_host_submit(tlr_ctx* ctx, const void* h_bf16_host, int32_t 
     const size_t bytes = nn * ctx->d * 2;
     cudaPointerAttributes attr;
     const void* mapped = nullptr;
-    // Above a few MB the copy engine is faster than the copy kernel and there is nothing left to hide.
-    if (bytes <= (4u << 20) && (bytes & 15u) == 0 && (reinterpret_cast<uintptr_t>(h_bf16_host) & 15u) == 0 &&
-        cudaPointerGetAttributes(&attr, h_bf16_host) == cudaSuccess && attr.type == cudaMemoryTypeHost)
+    bool pinned = false;
+    if (cudaPointerGetAttributes(&attr, h_bf16_host) == cudaSuccess && attr.type == cudaMemoryTypeHost) {
+      pinned = true;
       mapped = attr.devicePointer;
+    }
     cudaGetLastError();
-    if (mapped != nullptr) {
+    // Above a few MB the copy engine is faster than the copy kernel and there is nothing left to hide.
+    const bool by_kernel = mapped != nullptr && bytes <= (4u << 20) && (bytes & 15u) == 0 &&
+                           (reinterpret_cast<uintptr_t>(h_bf16_host) & 15u) == 0;
+    if (by_kernel) {
       if (tlr::launch_host_copy(mapped, ctx->h_stage[q], bytes, stream) != cudaSuccess) return TLR_ERR_CUDA;
+    } else if (pinned) {
+      // A large pinned batch: the copy engine brings it in on the context's own stream, beside the kernels of
+      // the call before it (this slot's last user has been collected, so its staging buffer is free), and the
+      // call's stream waits for the transfer only.
+      if (cudaMemcpyAsync(ctx->h_stage[q], h_bf16_host, bytes, cudaMemcpyHostToDevice, ctx->copy_stream) != cudaSuccess ||
+          cudaEventRecord(ctx->copy_done[q], ctx->copy_stream) != cudaSuccess ||
+          cudaStreamWaitEvent(stream, ctx->copy_done[q], 0) != cudaSuccess)
+        return TLR_ERR_CUDA;
     } else if (cudaMemcpyAsync(ctx->h_stage[q], h_bf16_host, bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) {
       return TLR_ERR_CUDA;
     }

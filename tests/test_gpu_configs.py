@@ -110,22 +110,23 @@ def test_config_sweep(pkg, n):
         check_against_oracle(O.with_threshold(scores, tau), gpu, h64, W64)
 
 
-def test_host_calls_in_flight_at_full_size(pkg):
-    """The decode batch of the benchmark through submit / collect with two calls in flight: the copy of the next
-    call's h overlaps the kernels of the call before it, so every collected result must still belong to ITS batch.
-    Four different batches (two sizes) go round 48 times; each collected result is compared bit for bit with the
-    device-buffer call on the same batch, and one batch of each size with the oracle."""
+@pytest.mark.parametrize("sizes,calls", [([256, 16, 256, 200], 48), ([2400, 1100, 4096, 3000], 10)])
+def test_host_calls_in_flight_at_full_size(pkg, sizes, calls):
+    """Batches through submit / collect with two calls in flight: the transfer of the next call's h (a copy kernel
+    for decode batches, the copy engine on the context's own stream for batches of several MB) overlaps the kernels
+    of the call before it, so every collected result must still belong to ITS batch.  Four different batches go
+    round; each collected result is compared bit for bit with the device-buffer call on the same batch, and two
+    of the batches with the oracle."""
     wl = S.WORKLOADS["decode256"]
     W, W64, Wd = Head.get(wl.d, wl.V)
-    sizes = [256, 16, 256, 200]
     hs = [S.make_h(n, wl.d, seed=40 + i).h for i, n in enumerate(sizes)]
     pinned = [h.pin_memory() for h in hs]
-    want = [run_gpu(pkg, Wd, h, wl.tau, max_n=256) for h in hs]
+    m = max(sizes)
+    want = [run_gpu(pkg, Wd, h, wl.tau, max_n=m) for h in hs]
     for i in (0, 1):
         ref = O.route_oracle(S.bf16_bits(hs[i]), S.bf16_bits(W), wl.tau, W64=W64)
         check_against_oracle(ref, want[i], O.bf16_bits_to_f64(S.bf16_bits(hs[i])), W64)
-    ctx = pkg.tlr_create(wl.d, wl.V, Wd, 256)
-    m = 256
+    ctx = pkg.tlr_create(wl.d, wl.V, Wd, m)
     outs = [(torch.empty(m, dtype=torch.int32).pin_memory(), torch.empty(m).pin_memory(), torch.empty(m).pin_memory(),
              torch.empty(m, dtype=torch.uint8).pin_memory(), torch.full((m,), -1, dtype=torch.int32).pin_memory(),
              torch.full((1,), -9, dtype=torch.int32).pin_memory()) for _ in range(2)]
@@ -139,7 +140,6 @@ def test_host_calls_in_flight_at_full_size(pkg):
         assert np.array_equal(o[1].numpy()[:n], w["conf"]) and np.array_equal(o[2].numpy()[:n], w["entropy"])
         assert np.array_equal(o[4].numpy()[:c], w["routed_idx"][:c])
 
-    calls = 48
     pkg.tlr_route_host_submit(ctx, pinned[0], sizes[0], wl.tau)
     for i in range(1, calls):
         pkg.tlr_route_host_submit(ctx, pinned[i % len(sizes)], sizes[i % len(sizes)], wl.tau)
